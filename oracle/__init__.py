@@ -61,6 +61,11 @@ def lib() -> C.CDLL:
         L.fosgd_oracle_flatten_entry.argtypes = [f64p, i64, cint, u64, u64, u32, i64]
         L.fosgd_oracle_flatten_entry.restype = dbl
         L.fosgd_oracle_encode.argtypes = [f64p, i64, cint, u64, u64, u32, dbl, cint, u32p, f32p]
+        i64p = C.POINTER(C.c_int64)
+        L.fosgd_oracle_decode_entry.argtypes = [u32p, i64, cint, u64, u64, u32, dbl, cint, i64]
+        L.fosgd_oracle_decode_entry.restype = dbl
+        L.fosgd_oracle_flatten_grid.argtypes = [C.c_void_p, cint, i64, u64, u64, u32, cint, i64p, cint, i64p, cint, f64p]
+        L.fosgd_oracle_decode_grid.argtypes = [u32p, i64, u64, u64, u32, dbl, cint, cint, i64p, cint, i64p, cint, f64p]
         L.fosgd_oracle_decode_full.argtypes = [u32p, i64, cint, u64, u64, u32, dbl, cint, f64p]
         L.fosgd_oracle_encode_tab.argtypes = [f64p, i64, cint, u64, u64, u32, f64p, cint, u32p, f32p]
         L.fosgd_oracle_decode_full_tab.argtypes = [u32p, i64, cint, u64, u64, u32, f64p, cint, f64p]
@@ -145,6 +150,39 @@ def flatten_entry(g, seed, step, wid, k, block_log2=0) -> float:
     g = _f64(g)
     return lib().fosgd_oracle_flatten_entry(_p(g, C.c_double), g.size, block_log2, seed, step,
                                             wid, k)
+
+
+def decode_entry(pl, d, seed, step, wid, lam_, k, K=1, block_log2=0) -> float:
+    """One output of the decoder (Def. 3.8) from the matrix definition."""
+    pl = _u32(pl)
+    return lib().fosgd_oracle_decode_entry(_p(pl, C.c_uint32), d, block_log2, seed, step, wid, lam_, K, k)
+
+
+def _grid(k_hi, k_lo):
+    hi, lo = np.ascontiguousarray(k_hi, dtype=np.int64), np.ascontiguousarray(k_lo, dtype=np.int64)
+    return hi, lo, np.empty((hi.size, lo.size), np.float64)
+
+
+def flatten_grid(g, seed, step, wid, split_log2, k_hi, k_lo) -> np.ndarray:
+    """Entries k = k_hi[a] * 2^split_log2 + k_lo[b] of the global transform H D_eps x -> [n_hi, n_lo].
+    g: float64, or float32 (used as is, for vectors too long to hold twice in host memory)."""
+    g = np.ascontiguousarray(g)
+    if g.dtype != np.float32:
+        g = _f64(g)
+    hi, lo, out = _grid(k_hi, k_lo)
+    lib().fosgd_oracle_flatten_grid(g.ctypes.data_as(C.c_void_p), int(g.dtype == np.float32), g.size, seed, step,
+                                    wid, split_log2, _p(hi, C.c_int64), hi.size, _p(lo, C.c_int64), lo.size,
+                                    _p(out, C.c_double))
+    return out
+
+
+def decode_grid(pl, d, seed, step, wid, lam_, split_log2, k_hi, k_lo, K=1) -> np.ndarray:
+    """Entries k = k_hi[a] * 2^split_log2 + k_lo[b] of the global decoder (Def. 3.8) -> [n_hi, n_lo]."""
+    pl = _u32(pl)
+    hi, lo, out = _grid(k_hi, k_lo)
+    lib().fosgd_oracle_decode_grid(_p(pl, C.c_uint32), d, seed, step, wid, lam_, K, split_log2,
+                                   _p(hi, C.c_int64), hi.size, _p(lo, C.c_int64), lo.size, _p(out, C.c_double))
+    return out
 
 
 def _lam_table(lam_, dp, block_log2):

@@ -12,8 +12,10 @@
  * Pins (see tests/test_oracle_*.py): dense Sylvester matrix brute force, H H = d I, norm
  * preservation, one-hot flatness (Def. 3.4), Lemma A.4 (mean = clip, MSE closed form),
  * Lemma A.5, Remark 5.2 (norm of the K=1 composite is exactly lambda sqrt(d')), Cor. A.8
- * variance of the N-worker average, Theorem 5.5 amplitude law, and the published
- * Philox4x32-10 known-answer vectors.
+ * variance of the N-worker average, the K-dither error bound of Lemma A.9, Theorem 5.5
+ * amplitude law, and the published Philox4x32-10 known-answer vectors.  The single-entry and
+ * product-grid functions (flatten_entry, decode_entry, flatten_grid, decode_grid) are pinned to
+ * the dense matrix and to the full transforms.
  *
  * Parity unpinned by the paper (readings taken where it is silent): zero padding to a
  * power of two and the blocked variant; the index-to-counter mapping of the generator; the
@@ -233,6 +235,122 @@ void fosgd_oracle_decode_full(const uint32_t* planes, int64_t d, int block_log2,
     for (int64_t b = 0; b < dp; b += n) fosgd_oracle_fwht(out + b, n);
     for (int64_t i = 0; i < dp; ++i)
         out[i] *= s * (double)fosgd_oracle_eps(seed, step, id, i);
+}
+
+/* One entry of the decoder of Def. 3.8 straight from the matrix definition
+ * H[k][j] = (-1)^popcount(k&j)/sqrt(n): out_k = (lambda / K) eps_k sum_j H[k][j] (2 c_j - K), the sum
+ * running over the block of k.  The twin of fosgd_oracle_flatten_entry for the decode side: it
+ * checks single outputs of decoders too long to run in full. */
+double fosgd_oracle_decode_entry(const uint32_t* planes, int64_t d, int block_log2, uint64_t seed,
+                                 uint64_t step, uint32_t id, double lambda, int K, int64_t k)
+{
+    int64_t dp = fosgd_oracle_padded_dim(d, block_log2);
+    int64_t n = transform_len(dp, block_log2);
+    int P = planes_for(K);
+    int64_t words = dp / 32;
+    int64_t b0 = (k / n) * n, kk = k - b0;
+    double acc = 0.0;   /* a sum of integers below 2^53: exact */
+    for (int64_t j = 0; j < n; ++j) {
+        int64_t i = b0 + j;
+        int c = 0;
+        for (int p = 0; p < P; ++p)
+            c |= (int)((planes[(int64_t)p * words + (i >> 5)] >> (i & 31)) & 1u) << p;
+        double q = (double)(2 * c - K);
+        acc += (__builtin_popcountll((unsigned long long)(kk & j)) & 1) ? -q : q;
+    }
+    return lambda / ((double)K * sqrt((double)n)) * (double)fosgd_oracle_eps(seed, step, id, k) * acc;
+}
+
+/* Entries of one global transform (block_log2 = 0, length n = d') on a product grid of output
+ * indices k = k_hi[a] 2^s + k_lo[b].  The recursion H_k = H_1 (x) H_{k-1} below Def. 3.4, applied
+ * to the top log2(n) - s index bits, reads H_n = H_{n / 2^s} (x) H_{2^s}, i.e. with j = j_hi 2^s + j_lo
+ *     (H v)[k_hi 2^s + k_lo] = n^{-1/2} sum_{j_hi} (-1)^popcount(k_hi & j_hi)
+ *                                       [ sum_{j_lo} (-1)^popcount(k_lo & j_lo) v_j ],
+ * so the bracket is shared by all k_hi and the whole grid costs n * n_lo multiply-adds instead of
+ * n * n_hi * n_lo.  The signs (-1)^popcount(k_lo & j_lo) are tabulated once as +-1.0.  Nothing
+ * else is reordered; both functions below are pinned to the single-entry functions above and to
+ * the full transforms.  out: [n_hi][n_lo]. */
+static double* walsh_sign_table(const int64_t* k_lo, int n_lo, int64_t lo_len)
+{
+    double* tab = (double*)malloc(sizeof(double) * (size_t)n_lo * (size_t)lo_len);
+    for (int64_t j_lo = 0; j_lo < lo_len; ++j_lo)
+        for (int b = 0; b < n_lo; ++b)
+            tab[j_lo * n_lo + b] =
+                (__builtin_popcountll((unsigned long long)(k_lo[b] & j_lo)) & 1) ? -1.0 : 1.0;
+    return tab;
+}
+
+/* sum over j_hi of +-inner (the outer Kronecker factor), for every k_hi of the grid */
+static void grid_outer(const double* inner, int64_t j_hi, const int64_t* k_hi, int n_hi, int n_lo,
+                       double* out)
+{
+    for (int a = 0; a < n_hi; ++a) {
+        int neg = __builtin_popcountll((unsigned long long)(k_hi[a] & j_hi)) & 1;
+        for (int b = 0; b < n_lo; ++b) out[a * n_lo + b] += neg ? -inner[b] : inner[b];
+    }
+}
+
+/* flatten_grid: v = D_eps x, x the zero-padded gradient, given as doubles (g_is_f32 = 0) or
+ * floats (g_is_f32 = 1, for vectors too long to hold twice in host memory). */
+void fosgd_oracle_flatten_grid(const void* g, int g_is_f32, int64_t d, uint64_t seed, uint64_t step,
+                               uint32_t id, int s, const int64_t* k_hi, int n_hi,
+                               const int64_t* k_lo, int n_lo, double* out)
+{
+    int64_t n = fosgd_oracle_padded_dim(d, 0);
+    int64_t lo_len = (int64_t)1 << s, hi_len = n >> s;
+    double* sgn = walsh_sign_table(k_lo, n_lo, lo_len);
+    double* inner = (double*)malloc(sizeof(double) * (size_t)n_lo);
+    for (int a = 0; a < n_hi * n_lo; ++a) out[a] = 0.0;
+    for (int64_t j_hi = 0; j_hi < hi_len; ++j_hi) {
+        for (int b = 0; b < n_lo; ++b) inner[b] = 0.0;
+        for (int64_t j_lo = 0; j_lo < lo_len; ++j_lo) {
+            int64_t j = j_hi * lo_len + j_lo;
+            if (j >= d) break;   /* padding: zeros from here to the end of the vector */
+            double x = g_is_f32 ? (double)((const float*)g)[j] : ((const double*)g)[j];
+            double v = (double)fosgd_oracle_eps(seed, step, id, j) * x;
+            const double* sj = sgn + j_lo * n_lo;
+            for (int b = 0; b < n_lo; ++b) inner[b] += sj[b] * v;
+        }
+        grid_outer(inner, j_hi, k_hi, n_hi, n_lo, out);
+    }
+    double sc = 1.0 / sqrt((double)n);
+    for (int a = 0; a < n_hi * n_lo; ++a) out[a] *= sc;
+    free(inner);
+    free(sgn);
+}
+
+/* decode_grid: the decoder of Def. 3.8 on the same kind of grid, v_j = 2 c_j - K read from the
+ * bit planes; every entry is scaled by lambda / (K sqrt n) and flipped by eps at its own index. */
+void fosgd_oracle_decode_grid(const uint32_t* planes, int64_t d, uint64_t seed, uint64_t step,
+                              uint32_t id, double lambda, int K, int s, const int64_t* k_hi,
+                              int n_hi, const int64_t* k_lo, int n_lo, double* out)
+{
+    int64_t n = fosgd_oracle_padded_dim(d, 0);
+    int64_t lo_len = (int64_t)1 << s, hi_len = n >> s;
+    int P = planes_for(K);
+    int64_t words = n / 32;
+    double* sgn = walsh_sign_table(k_lo, n_lo, lo_len);
+    double* inner = (double*)malloc(sizeof(double) * (size_t)n_lo);
+    for (int a = 0; a < n_hi * n_lo; ++a) out[a] = 0.0;
+    for (int64_t j_hi = 0; j_hi < hi_len; ++j_hi) {
+        for (int b = 0; b < n_lo; ++b) inner[b] = 0.0;
+        for (int64_t j_lo = 0; j_lo < lo_len; ++j_lo) {
+            int64_t j = j_hi * lo_len + j_lo;
+            int c = 0;
+            for (int p = 0; p < P; ++p)
+                c |= (int)((planes[(int64_t)p * words + (j >> 5)] >> (j & 31)) & 1u) << p;
+            double v = (double)(2 * c - K);
+            const double* sj = sgn + j_lo * n_lo;
+            for (int b = 0; b < n_lo; ++b) inner[b] += sj[b] * v;
+        }
+        grid_outer(inner, j_hi, k_hi, n_hi, n_lo, out);
+    }
+    double sc = lambda / ((double)K * sqrt((double)n));
+    for (int a = 0; a < n_hi; ++a)
+        for (int b = 0; b < n_lo; ++b)
+            out[a * n_lo + b] *= sc * (double)fosgd_oracle_eps(seed, step, id, k_hi[a] * lo_len + k_lo[b]);
+    free(inner);
+    free(sgn);
 }
 
 /* Blocked mode with one amplitude per block: Defs. 3.7 and 3.8 hold for each block of n = 2^b

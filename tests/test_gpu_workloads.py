@@ -1,8 +1,9 @@
 """Parity on the five benchmark workloads at full size, in the launch configuration bench.py
 times (all workers of a config in one call where they fit).  Configs 0-3: every bit and every
-averaged coordinate against the oracle.  Config 4 (d = 1.3e9, d' = 2^31): sampled transform
-outputs and bits that the oracle computes one by one from the matrix definition, plus
-properties that hold at any size (norm preservation, Remark 5.2's exact norm)."""
+averaged coordinate against the oracle.  Config 4 (d = 1.3e9, d' = 2^31): for workers 0, 1, 31 and
+63, sampled transform outputs, uplink bits, entries of the 4-worker average, downlink planes and
+downlink decoder outputs that the oracle computes from the matrix definition, plus properties
+that hold at any size (norm preservation, Remark 5.2's exact norm)."""
 import numpy as np
 import pytest
 import torch
@@ -83,18 +84,21 @@ def test_config3_resnet50_full_round_trip(F, block_log2):
     full_round_trip(F, synthetic.WORKLOADS[3], block_log2=block_log2)
 
 
-def test_two_strided_passes_2p26(F):
-    # L = 26 is the smallest length that needs two strided passes
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_two_strided_passes_2p26(F, dtype):
+    # L = 26 is the smallest length that needs two strided passes; every output, bit and decoded
+    # coordinate against the oracle, for both input types
     d, seed, step = (1 << 26) - 12345, 5, 6
-    g = torch.randn(1, d + 1, generator=torch.Generator(device=DEV).manual_seed(1), device=DEV)
+    stride = d + 1 if dtype == torch.float32 else d + 1 + 8 - (d + 1) % 8
+    g = torch.randn(1, stride, generator=torch.Generator(device=DEV).manual_seed(1), device=DEV).to(dtype)
     dp = F.padded_dim(d)
     ws = torch.empty(F.workspace_bytes(F.OP_ENCODE, d), dtype=torch.uint8, device=DEV)
     y = torch.empty(1, dp, dtype=torch.float32, device=DEV)
-    F.flatten(g, d, y, seed, step, ws=ws, worker_stride=d + 1)
+    F.flatten(g, d, y, seed, step, ws=ws, worker_stride=stride)
     gh = g[0, :d].cpu().double().numpy()
     lam = oracle.lam(float(np.linalg.norm(gh)), 2.0, dp)
     bits = torch.zeros(1, dp // 32, dtype=torch.int32, device=DEV)
-    F.encode(g, d, bits, lam, seed, step, ws=ws, worker_stride=d + 1)
+    F.encode(g, d, bits, lam, seed, step, ws=ws, worker_stride=stride)
     out = torch.empty(d, dtype=torch.float32, device=DEV)
     F.decode(bits[0], d, out, lam, seed, step, 0, ws=ws)
     torch.cuda.synchronize()
@@ -104,62 +108,166 @@ def test_two_strided_passes_2p26(F):
     assert_l2_close(out.cpu().numpy(), oracle.decode_full(to_np_words(bits)[0], d, seed, step, 0, lam)[:d])
 
 
+# ---- config 4 (d = 1.3e9, bf16, 64 workers): sampled coordinates at full size --------------------
+CFG4_WORKERS = (0, 1, 31, 63)
+GRID_SPLIT = 12          # global mode: samples k = k_hi * 2^12 + k_lo
+
+
+def cfg4_sample_grid(dp, rng):
+    """Global mode (d' = 2^31, passes over index bits [0,11), [11,21), [21,31)): a product grid of
+    32 x 16 = 512 coordinates.  k_lo takes every value of the low five bits (the lane / packed-bit
+    position) once, with bits 5..11 running through all-zero, all-one (both ends of a contiguous
+    tile), single bits and random patterns; k_hi does the same for the bits of the two strided
+    passes."""
+    low5 = rng.permutation(32)
+    mid7 = np.concatenate([[0, 127, 63, 64, 1, 2, 4, 8, 16, 32], rng.integers(0, 128, 22)])
+    k_lo = (mid7 << 5) | low5
+    nhi = dp >> GRID_SPLIT
+    k_hi = np.concatenate([[0, nhi - 1, 1, nhi >> 1, (nhi >> 1) - 1, 1 << 9, (1 << 9) - 1, 1 << 8],
+                           rng.integers(0, nhi, 8)])
+    return k_hi.astype(np.int64), k_lo.astype(np.int64)
+
+
+def grid_in_threads(fn, k_hi, k_lo, parts=4):
+    """fn(k_hi, k_lo_part) -> [n_hi, len(part)], the k_lo set cut into parts that run side by side."""
+    cols = pmap(lambda c: fn(k_hi, c), np.array_split(k_lo, parts))
+    return np.concatenate(cols, axis=1)
+
+
+def assert_sampled_bits(words, ks, y_ref, lam, seed, step, wid, K=1, plane_words=None):
+    """Bits (K = 1) or count planes of the sampled coordinates against sign(y + tau_k), wherever the
+    oracle's decision is not inside the tie band."""
+    ties = 0
+    for idx, (k, yr) in enumerate(zip(ks, y_ref)):
+        zs = [yr + lam * oracle.dither_t(seed, step, wid, kk, int(k)) / 2.0 ** 24 for kk in range(K)]
+        if min(abs(z) for z in zs) <= 1e-5 * lam:
+            ties += 1
+            continue
+        c = sum(1 for z in zs if z >= 0)
+        got = sum(((int(words[p][idx]) >> (int(k) & 31)) & 1) << p for p in range(len(words)))
+        assert got == c, (int(k), got, c)
+    assert ties <= max(2, len(ks) // 100)
+    return ties
+
+
 @pytest.mark.parametrize("block_log2", [0, 20])
 def test_config4_bf16_1p3B_sampled(F, block_log2):
+    """Config 4 at full size: the transform, the uplink bits, the 4-worker server average, the downlink
+    planes and the downlink decoder, each on 512 coordinates per worker that the oracle computes from
+    the matrix definition (global mode: on a product grid; blocked mode: entry by entry), plus the
+    properties that hold at any size."""
     from paper_2405_11095_b200 import synthetic
     w = synthetic.WORKLOADS[4]
-    d, seed, step = w.d, 77, 1
-    dp = F.padded_dim(d, block_log2)
-    n_eff = F.transform_len(d, block_log2)
-    ws = torch.empty(F.workspace_bytes(F.OP_AGGREGATE, d, block_log2=block_log2), dtype=torch.uint8, device=DEV)
+    d, seed, step, K = w.d, 77, 1, w.K
+    b = block_log2
+    dp = F.padded_dim(d, b)
+    n_eff = F.transform_len(d, b)
+    P = F.planes(K)
+    ws = torch.empty(F.workspace_bytes(F.OP_AGGREGATE, d, block_log2=b), dtype=torch.uint8, device=DEV)
     g = torch.empty(1, d, dtype=torch.bfloat16, device=DEV)
     y = torch.empty(1, dp, dtype=torch.float32, device=DEV)
-    bits = torch.zeros(2, dp // 32, dtype=torch.int32, device=DEV)
-    acc = torch.empty(dp, dtype=torch.float32, device=DEV)
-    rng = np.random.default_rng(4)
-    workers = (0, 63)
+    bits = torch.zeros(len(CFG4_WORKERS), dp // 32, dtype=torch.int32, device=DEV)
+    rng = np.random.default_rng(4 + b)
+    if b == 0:
+        k_hi, k_lo = cfg4_sample_grid(dp, rng)
+        ks = (k_hi[:, None] * (1 << GRID_SPLIT) + k_lo[None, :]).reshape(-1)
+    else:
+        blk = 1 << b
+        ks = np.concatenate([rng.integers(0, dp, 480), [0, 31, 32, 1023, 1024, blk - 1, blk, dp - blk, dp - 1],
+                             (dp - blk) + rng.integers(0, blk, 23)]).astype(np.int64)
+    ks_dev = torch.from_numpy(ks).to(DEV)
     lam = None
-    for slot, n in enumerate(workers):
+    for slot, n in enumerate(CFG4_WORKERS):
         synthetic.worker_gradient(w, n, DEV, out=g[0])
         norm = float(g.double().norm())
         if lam is None:
-            lam = F.lambda_(1.05 * norm, w.alpha, n_eff)      # an a-priori bound, same for both workers
-        F.flatten(g, d, y, seed, step, worker_id0=n, block_log2=block_log2, ws=ws)
-        F.encode(g, d, bits[slot:slot + 1], lam, seed, step, worker_id0=n, block_log2=block_log2, ws=ws)
+            lam = F.lambda_(1.05 * norm, w.alpha, n_eff)      # an a-priori bound, same for all workers
+        F.flatten(g, d, y, seed, step, worker_id0=n, block_log2=b, ws=ws)
+        F.encode(g, d, bits[slot:slot + 1], lam, seed, step, worker_id0=n, block_log2=b, ws=ws)
         torch.cuda.synchronize()
         # property at full size: H D_eps is orthonormal
         assert abs(float(y.double().norm()) / norm - 1) < 1e-5
-        # sampled outputs, each computed by the oracle from the matrix definition
-        gh = g[0].cpu().double().numpy()
-        idx = np.concatenate([rng.integers(0, dp, 3 if block_log2 == 0 else 48), [0, dp - 1]])
-        yv = y[0, torch.from_numpy(idx).to(DEV)].cpu().numpy()
-        wv = to_np_words(bits[slot, torch.from_numpy(idx >> 5).to(DEV)])
-        ref = np.array(pmap(lambda k: oracle.flatten_entry(gh, seed, step, n, int(k), block_log2=block_log2), idx))
+        yv = y[0, ks_dev].cpu().double().numpy()
+        wv = to_np_words(bits[slot, ks_dev >> 5])
         scale = float(y.abs().max())
-        assert np.abs(yv - ref).max() <= 1e-5 * scale
-        for k, yr, word in zip(idx, ref, wv):
-            z = yr + lam * oracle.dither_t(seed, step, n, 0, int(k)) / 2.0 ** 24
-            if abs(z) > 1e-5 * lam:
-                assert ((int(word) >> (int(k) & 31)) & 1) == (1 if z >= 0 else 0)
+        gh = g[0].float().cpu().numpy()                       # bf16 -> fp32 is exact
+        if b == 0:
+            ref = grid_in_threads(lambda hi, lo: oracle.flatten_grid(gh, seed, step, n, GRID_SPLIT, hi, lo),
+                                  k_hi, k_lo).reshape(-1)
+        else:
+            gd = gh.astype(np.float64)
+            ref = np.array(pmap(lambda k: oracle.flatten_entry(gd, seed, step, n, int(k), block_log2=b), ks))
+            del gd
         del gh
-    # streamed aggregation of the two workers into one accumulator: chunk by chunk == Remark 5.2 checks
-    F.server_aggregate(bits[0:1], d, acc, lam, seed, step, N_total=1, worker_id0=workers[0], block_log2=block_log2, ws=ws)
+        assert np.abs(yv - ref).max() <= 1e-5 * scale
+        assert np.linalg.norm(yv - ref) <= 1e-5 * np.linalg.norm(ref)
+        assert_sampled_bits([wv], ks, ref, lam, seed, step, n)
+    del y, g
+
+    # ---- server: the four workers in three chunks into one accumulator, then the downlink encoder ----
+    lam_s = F.lambda_server(lam, w.alpha_s, n_eff)
+    acc = torch.empty(dp, dtype=torch.float32, device=DEV)
+    down = torch.zeros(P, dp // 32, dtype=torch.int32, device=DEV)
+    N = len(CFG4_WORKERS)
+    F.server_aggregate(bits[0:2], d, acc, lam, seed, step, N_total=N, worker_id0=0, flags=F.AGG_BEGIN,
+                       block_log2=b, ws=ws)
+    F.server_aggregate(bits[2:3], d, acc, lam, seed, step, N_total=N, worker_id0=31, flags=0, block_log2=b, ws=ws)
+    F.server_aggregate(bits[3:4], d, acc, lam, seed, step, N_total=N, worker_id0=63, flags=F.AGG_END,
+                       lam_s=lam_s, K=K, down_bits=down, block_log2=b, ws=ws)
+    out = torch.empty(d, dtype=torch.float32, device=DEV)
+    F.downlink_decode(down, d, out, lam_s, seed, step, K=K, block_log2=b, ws=ws)
     torch.cuda.synchronize()
-    assert abs(float(acc.double().norm()) / (lam * np.sqrt(dp)) - 1) < 1e-5      # ||D(q)|| = lambda sqrt(d')
-    one = acc.clone()
-    F.server_aggregate(bits[0:1], d, acc, lam, seed, step, N_total=2, worker_id0=workers[0], flags=F.AGG_BEGIN,
-                       block_log2=block_log2, ws=ws)
-    F.server_aggregate(bits[1:2], d, acc, lam, seed, step, N_total=2, worker_id0=workers[1], flags=F.AGG_END,
-                       block_log2=block_log2, ws=ws)
-    two = acc.clone()
-    F.server_aggregate(bits[1:2], d, acc, lam, seed, step, N_total=1, worker_id0=workers[1], block_log2=block_log2, ws=ws)
+    # ||gbar|| <= lambda sqrt(d') (Remark 5.2 and the triangle inequality)
+    assert float(acc.double().norm()) <= lam * np.sqrt(dp) * (1 + 1e-5)
+    bw = to_np_words(bits)
+    if b == 0:
+        parts = [grid_in_threads(lambda hi, lo, s=slot, n=n: oracle.decode_grid(bw[s], d, seed, step, n, lam,
+                                                                                GRID_SPLIT, hi, lo), k_hi, k_lo, parts=2)
+                 for slot, n in enumerate(CFG4_WORKERS)]
+        gbar_ref = np.mean(parts, axis=0).reshape(-1)
+    else:
+        gbar_ref = np.mean([pmap(lambda k, s=slot, n=n: oracle.decode_entry(bw[s], d, seed, step, n, lam, int(k),
+                                                                            block_log2=b), ks)
+                            for slot, n in enumerate(CFG4_WORKERS)], axis=0)
+    accv = acc[ks_dev].cpu().double().numpy()
+    assert np.linalg.norm(accv - gbar_ref) <= 1e-5 * np.linalg.norm(gbar_ref)
+    assert np.abs(accv - gbar_ref).max() <= 1e-5 * np.abs(gbar_ref).max()
+    del bw
+
+    # downlink planes: the oracle's transform of the accumulator the GPU holds (the encoder's input)
+    acch = acc.cpu().numpy()
+    if b == 0:
+        ys = grid_in_threads(lambda hi, lo: oracle.flatten_grid(acch, seed, step, oracle.SERVER_ID, GRID_SPLIT, hi, lo),
+                             k_hi, k_lo).reshape(-1)
+    else:
+        accd = acch.astype(np.float64)
+        ys = np.array(pmap(lambda k: oracle.flatten_entry(accd, seed, step, oracle.SERVER_ID, int(k), block_log2=b), ks))
+        del accd
+    del acch
+    dwords = [to_np_words(down[p, ks_dev >> 5]) for p in range(P)]
+    assert_sampled_bits(dwords, ks, ys, lam_s, seed, step, oracle.SERVER_ID, K=K)
+
+    # downlink decoder on the planes the GPU produced, coordinates below d
+    dw = to_np_words(down)
+    keep = ks < d
+    if b == 0:
+        ref_out = grid_in_threads(lambda hi, lo: oracle.decode_grid(dw, dp, seed, step, oracle.SERVER_ID, lam_s,
+                                                                    GRID_SPLIT, hi, lo, K=K), k_hi, k_lo).reshape(-1)[keep]
+    else:
+        ref_out = np.array(pmap(lambda k: oracle.decode_entry(dw, dp, seed, step, oracle.SERVER_ID, lam_s, int(k),
+                                                              K=K, block_log2=b), ks[keep]))
+    outv = out[ks_dev[torch.from_numpy(keep).to(DEV)]].cpu().double().numpy()
+    assert keep.sum() >= 200
+    assert np.linalg.norm(outv - ref_out) <= 1e-5 * np.linalg.norm(ref_out)
+    # the decoded average is an unbiased estimate of the mean gradient: <Z, x> / ||x||^2 ~ 1 for worker 63
+    g = torch.empty(d, dtype=torch.bfloat16, device=DEV)
+    synthetic.worker_gradient(w, CFG4_WORKERS[-1], DEV, out=g)
+    x = g.double()
+    one = torch.empty(dp, dtype=torch.float32, device=DEV)
+    F.server_aggregate(bits[3:4], d, one, lam, seed, step, N_total=1, worker_id0=63, block_log2=b, ws=ws)
     torch.cuda.synchronize()
-    err = float((two.double() - 0.5 * (one.double() + acc.double())).norm() / two.double().norm())
-    assert err < 1e-5
-    # the decoded vector is an unbiased estimate of the gradient: <Z(x), x> / ||x||^2 ~ 1
-    synthetic.worker_gradient(w, workers[1], DEV, out=g[0])
-    x = g[0].double()
-    ratio = float((acc[:d].double() * x).sum() / (x * x).sum())
+    assert abs(float(one.double().norm()) / (lam * np.sqrt(dp)) - 1) < 1e-5      # Remark 5.2: ||D(q)|| = lambda sqrt(d')
+    ratio = float((one[:d].double() * x).sum() / (x * x).sum())
     assert abs(ratio - 1) < 0.05
 
 

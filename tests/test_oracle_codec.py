@@ -258,3 +258,101 @@ def test_block_amplitude_law():
     # the flattening event of Lemma 3.6 per block: no transformed entry exceeds its block's lambda
     y = oracle.flatten(G[0], 1, 2, 0, block_log2=b).reshape(6, n)
     assert (np.abs(y).max(axis=1) <= lam[0] + 1e-300).all()
+
+
+def _dense_h(n):
+    i = np.arange(n)
+    return np.where(np.array([[bin(a & b).count("1") & 1 for b in i] for a in i]), -1.0, 1.0) / np.sqrt(n)
+
+
+@pytest.mark.parametrize("K", [1, 3])
+def test_decode_entry_is_the_dense_matrix_row(K):
+    # Def. 3.8 entry by entry: (lambda/K) eps_k sum_j H[k][j] (2 c_j - K), against the dense matrix
+    # written out here and against the full decoder, in global and in blocked mode
+    n, lam = 128, 0.75
+    rng = np.random.default_rng(20 + K)
+    P = oracle.planes(K)
+    pl = rng.integers(0, 2 ** 32, (P, n // 32), dtype=np.uint64).astype(np.uint32)
+    if P == 2:
+        pl[1] &= ~pl[0] | rng.integers(0, 2 ** 32, n // 32, dtype=np.uint64).astype(np.uint32)   # counts 0..3
+    c = sum(oracle.unpack(pl[p], n).astype(int) << p for p in range(P))
+    q = 2.0 * c - K
+    e = oracle.eps_vector(6, 7, 8, n)
+    dense = lam / K * e * (_dense_h(n) @ q)
+    full = oracle.decode_full(pl, n, 6, 7, 8, lam, K=K)
+    for k in range(n):
+        v = oracle.decode_entry(pl, n, 6, 7, 8, lam, k, K=K)
+        assert abs(v - dense[k]) <= 1e-13
+        assert abs(v - full[k]) <= 1e-13
+    # blocked mode: the sum runs over the block of k only, d not a multiple of the block
+    d, b = 200, 6
+    dp = oracle.padded_dim(d, b)
+    plb = rng.integers(0, 2 ** 32, (1, dp // 32), dtype=np.uint64).astype(np.uint32)
+    fullb = oracle.decode_full(plb, d, 1, 2, 3, lam, block_log2=b)
+    Hb = _dense_h(1 << b)
+    eb = oracle.eps_vector(1, 2, 3, dp)
+    qb = signs(plb[0], dp)
+    for k in (0, 63, 64, 129, dp - 1):
+        blk = k >> b
+        ref = lam * eb[k] * (Hb[k & 63] @ qb[blk << b:(blk + 1) << b])
+        v = oracle.decode_entry(plb, d, 1, 2, 3, lam, k, block_log2=b)
+        assert abs(v - ref) <= 1e-13 and abs(v - fullb[k]) <= 1e-13
+
+
+@pytest.mark.parametrize("split", [1, 4, 7, 9])
+def test_grid_entries_match_full_transforms(split):
+    # the product-grid functions (Kronecker split of the Sylvester matrix at `split` bits) against the
+    # full transform, the single-entry functions and, for one small case, the dense matrix
+    d, seed, step, wid = 700, 3, 4, 5
+    dp = oracle.padded_dim(d)                         # 1024
+    rng = np.random.default_rng(split)
+    g = rng.standard_normal(d)
+    k_hi = np.unique(np.concatenate([[0, (dp >> split) - 1], rng.integers(0, dp >> split, 5)]))
+    k_lo = np.unique(np.concatenate([[0, (1 << split) - 1], rng.integers(0, 1 << split, 6)]))
+    y = oracle.flatten(g, seed, step, wid)
+    grid = oracle.flatten_grid(g, seed, step, wid, split, k_hi, k_lo)
+    grid32 = oracle.flatten_grid(g.astype(np.float32), seed, step, wid, split, k_hi, k_lo)
+    y32 = oracle.flatten(g.astype(np.float32).astype(np.float64), seed, step, wid)
+    x = np.zeros(dp)
+    x[:d] = g * oracle.eps_vector(seed, step, wid, d)
+    dense = _dense_h(dp) @ x
+    for a, kh in enumerate(k_hi):
+        for b, kl in enumerate(k_lo):
+            k = int(kh) * (1 << split) + int(kl)
+            assert abs(grid[a, b] - y[k]) <= 1e-12
+            assert abs(grid[a, b] - dense[k]) <= 1e-12
+            assert abs(grid[a, b] - oracle.flatten_entry(g, seed, step, wid, k)) <= 1e-12
+            assert abs(grid32[a, b] - y32[k]) <= 1e-12
+    for K in (1, 7):
+        P = oracle.planes(K)
+        pl = rng.integers(0, 2 ** 32, (P, dp // 32), dtype=np.uint64).astype(np.uint32)
+        lam = 0.3
+        full = oracle.decode_full(pl, d, seed, step, wid, lam, K=K)
+        gridd = oracle.decode_grid(pl, d, seed, step, wid, lam, split, k_hi, k_lo, K=K)
+        for a, kh in enumerate(k_hi):
+            for b, kl in enumerate(k_lo):
+                k = int(kh) * (1 << split) + int(kl)
+                assert abs(gridd[a, b] - full[k]) <= 1e-12
+                assert abs(gridd[a, b] - oracle.decode_entry(pl, d, seed, step, wid, lam, k, K=K)) <= 1e-12
+
+
+def test_k_dither_error_bound():
+    # Lemma A.9: for ||x|| <= B, lambda = alpha B sqrt(log d / d), alpha >= 2,
+    #   E||Z_{lambda,K}(x) - x||^2 <= alpha^2 B^2 log d / K + 8 B^2 exp(-alpha^2 log d / 8)
+    # (expectation over eps and the K dithers: the step number draws both afresh)
+    d, T, alpha = 256, 600, 2.0
+    rng = np.random.default_rng(12)
+    cases = [rng.standard_normal(d), np.eye(d)[17] * 3.0, np.where(rng.random(d) < 0.05, rng.standard_normal(d), 0.0)]
+    for x in cases:
+        B = np.linalg.norm(x)
+        lam = oracle.lam(B, alpha, d)
+        for K in (1, 3, 15):
+            errs = np.empty(T)
+            for step in range(T):
+                pl = oracle.encode(x, 61, step, 9, lam, K=K)
+                z = oracle.decode_full(pl, d, 61, step, 9, lam, K=K)
+                errs[step] = ((z - x) ** 2).sum()
+            bound = alpha ** 2 * B ** 2 * np.log(d) / K + 8 * B ** 2 * np.exp(-alpha ** 2 * np.log(d) / 8)
+            assert errs.mean() + 5 * errs.std() / np.sqrt(T) <= bound
+            # the first term is attained up to ||x||^2 / K when the flattened vector stays in range
+            assert errs.mean() >= 0.5 * (lam ** 2 * d - B ** 2) / K
