@@ -10,9 +10,11 @@
  *
  * Conventions shared by every entry point
  *   - All data pointers are DEVICE pointers owned by the caller.  The library allocates
- *     nothing and never synchronises: work is enqueued on `stream` and the call returns.  Its
- *     only state between calls is diagnostic (the last CUDA error and the trace hooks per host
- *     thread, the timeout counter per device) plus the built-in scratch of fosgd_decode_noalloc.
+ *     nothing and does not synchronise: work is enqueued on `stream` and the call returns
+ *     (the one exception is the health check fosgd_async_timeouts, which waits for the device).
+ *     Its only state between calls is diagnostic (the last CUDA error and the trace hooks per
+ *     host thread, the timeout counter per device) plus the built-in scratch of
+ *     fosgd_decode_noalloc.
  *   - d is the true gradient length; d' = fosgd_padded_dim(d, block_log2) is the length the
  *     transform runs on.  block_log2 = 0: one transform of length d' = next power of two
  *     (>= 32).  block_log2 = b in [5, 30]: independent transforms on consecutive blocks of
@@ -35,9 +37,11 @@
  *     the minimum (one worker in flight); the calls that take several workers batch as many
  *     per launch as a larger `ws` allows.  Transforms that fit one thread block's tile
  *     (length <= 2^15) need none (ws may be NULL, ws_bytes 0).
- *   - Return value: FOSGD_OK or a negative status.  On any error nothing has been
- *     enqueued.  FOSGD_ECUDA means a launch failed; fosgd_last_cuda_error() (thread local)
- *     returns the cudaError_t.
+ *   - Return value: FOSGD_OK or a negative status.  On an argument, alignment, workspace,
+ *     size or limit error (every status but FOSGD_ECUDA) nothing has been enqueued.
+ *     FOSGD_ECUDA means a launch or a runtime call failed, possibly after earlier kernels of
+ *     the same call were enqueued: outputs, scratch and the accumulator are then undefined;
+ *     fosgd_last_cuda_error() (thread local) returns the cudaError_t.
  */
 #ifndef FOSGD_H
 #define FOSGD_H
@@ -192,8 +196,12 @@ int fosgd_downlink_apply(const uint32_t* down_bits, int64_t d, uint64_t seed, ui
  * decode (no allocator reachable from their code, cudaMalloc banned because it synchronises,
  * or no memory left to ask for), the scratch is a fixed array of FOSGD_NOALLOC_SCRATCH_BYTES
  * inside the library image; every GPU that loads the library holds it until the process ends.
- *   - Limit: the padded length d' must not exceed 2^20 coordinates (the scratch holds d'
- *     floats); larger sizes return FOSGD_ELIMIT and enqueue nothing.
+ *   - Limit: the scratch that fosgd_workspace_bytes(FOSGD_OP_DECODE, ...) asks for must fit,
+ *     i.e. a decoder whose transform takes several passes (transform length above 2^15, in
+ *     global or blocked mode) is accepted up to d' = 2^20 coordinates (d' floats of scratch);
+ *     single-pass decoders need no scratch and are accepted at any size.  Beyond the limit the
+ *     call returns FOSGD_ELIMIT and enqueues nothing.  The decoder's own argument checks
+ *     (FOSGD_EINVAL, FOSGD_EALIGN) come first.
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call outside any stream capture.  Later calls only launch.
  *   - The call allocates nothing and frees nothing.
@@ -219,6 +227,17 @@ int fosgd_async_timeouts(int* count);
 int fosgd_trace_passes(void** events, int capacity);
 int fosgd_trace_count(void);            /* launches recorded since the array was set */
 const char* fosgd_trace_label(int k);   /* e.g. "col10:f32->ws@32", "row14:ws->pack1@32" (kernel, source->sink, workers); valid until the next call */
+
+/* Issue-rate probe (measurement aid; no counterpart in the paper).  Enqueues one kernel that
+ * keeps every scheduler of every SM busy with independent register-resident chains of one
+ * instruction kind: fp32 add, fp32 fused multiply-add, three-input integer logic, or 32-bit
+ * integer multiply-add.  *lane_ops (HOST pointer) receives the number of lane operations the
+ * kernel executes (threads x iters x operations per iteration); divided by the kernel's duration,
+ * timed by the caller with events on `stream`, it is the rate the plain ALUs sustain on this
+ * device at the clock it runs.  sink: DEVICE pointer to at least 4 writable bytes (never written
+ * in practice).  iters in [1, 2^24]. */
+enum { FOSGD_PROBE_FADD = 0, FOSGD_PROBE_FFMA = 1, FOSGD_PROBE_LOP3 = 2, FOSGD_PROBE_IMAD = 3 };
+int fosgd_probe_issue_rate(int kind, int iters, double* lane_ops, uint32_t* sink, fosgd_stream stream);
 
 const char* fosgd_strerror(int status);
 int fosgd_last_cuda_error(void);

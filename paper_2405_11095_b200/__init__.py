@@ -26,7 +26,7 @@ EXPORTS = ("fosgd_padded_dim", "fosgd_planes", "fosgd_lambda", "fosgd_lambda_ser
            "fosgd_last_cuda_error", "fosgd_version", "fosgd_trace_passes", "fosgd_trace_count",
            "fosgd_trace_label", "fosgd_decode_noalloc", "fosgd_async_timeouts", "fosgd_amplitudes",
            "fosgd_encode_dev", "fosgd_server_aggregate_dev", "fosgd_downlink_decode_dev", "fosgd_downlink_apply",
-           "fosgd_downlink_encode")
+           "fosgd_downlink_encode", "fosgd_probe_issue_rate")
 
 
 class FosgdError(RuntimeError):
@@ -66,6 +66,7 @@ def _load() -> C.CDLL:
     L.fosgd_downlink_encode.argtypes = [vp, i64, u64, u64, C.c_float, vp, cint, cint, cint, vp, vp, sz, vp]
     L.fosgd_downlink_apply.argtypes = [vp, i64, u64, u64, C.c_float, vp, cint, cint, cint, C.c_float, vp, vp, sz, vp]
     L.fosgd_downlink_decode_dev.argtypes = [vp, i64, u64, u64, vp, cint, cint, cint, vp, vp, sz, vp]
+    L.fosgd_probe_issue_rate.argtypes = [cint, cint, C.POINTER(dbl), vp, vp]
     L.fosgd_strerror.argtypes, L.fosgd_strerror.restype = [cint], C.c_char_p
     L.fosgd_last_cuda_error.restype = cint
     L.fosgd_version.restype = C.c_char_p
@@ -176,8 +177,8 @@ def decode(bits, d, out, lam, seed, step, worker_id, block_log2=0, ws=None):
 def decode_noalloc(bits, d, out, lam, seed, step, worker_id, block_log2=0):
     """fosgd_decode_noalloc: fosgd_decode for callers that cannot allocate device scratch.
 
-    The scratch is a fixed 4 MiB array inside the library (so d' <= 2^20, else ELIMIT); the
-    call allocates nothing.  Calls share that array: do not let two of them overlap on a GPU.
+    The scratch is a fixed 4 MiB array inside the library (multi-pass transforms up to d' = 2^20,
+    else ELIMIT; single-pass ones need none); the call allocates nothing.  Calls share that array: do not let two of them overlap on a GPU.
     The first call on a device should happen outside stream capture."""
     _check(_lib.fosgd_decode_noalloc(_ptr(bits), d, worker_id, seed, step, lam, block_log2, _ptr(out),
                                      _stream()), "fosgd_decode_noalloc")
@@ -261,6 +262,17 @@ def downlink_apply(down_bits, d, x, lam_s, seed, step, step_size, K=1, block_log
                                      _ptr(dev), int(per_block), K, block_log2, float(step_size), _ptr(x),
                                      _ptr(ws), _nbytes(ws), _stream()), "fosgd_downlink_apply")
     return x
+
+
+PROBE_FADD, PROBE_FFMA, PROBE_LOP3, PROBE_IMAD = range(4)
+
+
+def probe_issue_rate(kind: int, iters: int, sink) -> float:
+    """fosgd_probe_issue_rate: enqueue the probe kernel of `kind` on the current stream and return
+    the lane operations it executes (time it with events around this call)."""
+    ops = C.c_double(0.0)
+    _check(_lib.fosgd_probe_issue_rate(kind, iters, C.byref(ops), _ptr(sink), _stream()), "fosgd_probe_issue_rate")
+    return ops.value
 
 
 def async_timeouts() -> int:

@@ -282,6 +282,17 @@ int check_grad_args(const void* grads, int dtype, int64_t d, int64_t worker_stri
 }
 
 }  // namespace
+
+void set_last_cuda_error(int e) { g_last_cuda_error = e; }
+
+int check_decode_args(const void* bits, int64_t d, float lambda, int block_log2, const void* out)
+{
+    if (bits == nullptr || out == nullptr || d < 1 || !valid_block(block_log2) || !good_lambda(lambda))
+        return FOSGD_EINVAL;
+    if (!aligned16(bits) || !aligned16(out)) return FOSGD_EALIGN;
+    return padded_dim(d, block_log2) < 0 ? FOSGD_EUNSUPPORTED : FOSGD_OK;
+}
+
 }  // namespace fosgd
 
 using namespace fosgd;
@@ -381,9 +392,9 @@ int fosgd_decode(const uint32_t* bits, int64_t d, uint32_t worker_id, uint64_t s
                  float lambda, int block_log2, float* out, void* ws, size_t ws_bytes,
                  fosgd_stream stream)
 {
-    if (bits == nullptr || out == nullptr || d < 1 || !valid_block(block_log2) || !good_lambda(lambda))
-        return FOSGD_EINVAL;
-    if (!aligned16(bits) || !aligned16(out) || (ws && !aligned16(ws))) return FOSGD_EALIGN;
+    const int st = check_decode_args(bits, d, lambda, block_log2, out);
+    if (st != FOSGD_OK) return st;
+    if (ws && !aligned16(ws)) return FOSGD_EALIGN;
     Geometry g;
     if (!make_geometry(d, block_log2, &g)) return FOSGD_EUNSUPPORTED;
     PassParams p{};
@@ -579,7 +590,7 @@ const char* fosgd_strerror(int status)
         case FOSGD_EWORKSPACE: return "workspace missing or too small";
         case FOSGD_EUNSUPPORTED: return "unsupported dtype, op or size";
         case FOSGD_ECUDA: return "CUDA launch error (see fosgd_last_cuda_error)";
-        case FOSGD_ELIMIT: return "padded length exceeds the 2^20 coordinates of the built-in scratch";
+        case FOSGD_ELIMIT: return "scratch need exceeds the built-in array (multi-pass transforms: d' <= 2^20 coordinates)";
     }
     return "unknown status";
 }

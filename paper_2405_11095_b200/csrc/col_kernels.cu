@@ -278,6 +278,10 @@ __global__ void __launch_bounds__(1024, 1) col_tma16_kernel(const PassParams p, 
     constexpr int BUF_WORDS = (1 << A) * 16;
     extern __shared__ __align__(128) float smem[];
     uint64_t* const full = reinterpret_cast<uint64_t*>(smem + 3 * BUF_WORDS);
+    // Copies issued into / tiles taken out of each buffer (written by one thread of the issuing resp.
+    // consuming group), and the flag that stops all issuing once a bounded wait has given up: the
+    // block then drains what is still in flight before any of its threads exits.
+    __shared__ int s_issued[3], s_taken[3], s_stop;
 
     const int tid = threadIdx.x;
     const int g = tid >> 9;
@@ -289,7 +293,12 @@ __global__ void __launch_bounds__(1024, 1) col_tma16_kernel(const PassParams p, 
     const int64_t nitems = (total - (int64_t)blockIdx.x + gridDim.x - 1) / gridDim.x;
 
     if (tid == 0) {
-        for (int b = 0; b < 3; ++b) mbar_init(full + b, 1);
+        for (int b = 0; b < 3; ++b) {
+            mbar_init(full + b, 1);
+            s_issued[b] = 0;
+            s_taken[b] = 0;
+        }
+        s_stop = 0;
     }
     __syncthreads();
 
@@ -302,12 +311,14 @@ __global__ void __launch_bounds__(1024, 1) col_tma16_kernel(const PassParams p, 
     };
     // one thread: four box copies (256 rows x 16 columns each) into buffer j % 3
     auto issue = [&](int64_t j) {
+        if (*(volatile int*)&s_stop) return;
         int n;
         uint32_t lo0, hi;
         item_coords(j, n, lo0, hi);
         uint64_t* const bar = full + (j % 3);
         const uint32_t dst0 = smem_u32(smem + (j % 3) * BUF_WORDS);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        s_issued[j % 3] += 1;
+        fence_generic_before_async();
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(65536u) : "memory");
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -346,9 +357,13 @@ __global__ void __launch_bounds__(1024, 1) col_tma16_kernel(const PassParams p, 
         }
         // bounded wait; the group then agrees on the outcome, so that it stops as a whole
         if (!group_all(1 + g, GT, mbar_wait(full + (j % 3), (uint32_t)((j / 3) & 1)))) {
-            if (gt == 0) atomicAdd(&g_col_wait_timeouts, 1);
-            return;
+            if (gt == 0) {
+                atomicAdd(&g_col_wait_timeouts, 1);
+                *(volatile int*)&s_stop = 1;
+            }
+            break;
         }
+        if (gt == 0) s_taken[j % 3] += 1;
         if (SRC == SRC_G32) {
             // the map covers whole rows only: a last partial row of the gradient is patched in
             const uint32_t row_p = full_rows - (hi << A);                  // tile-local index of that row
@@ -376,6 +391,7 @@ __global__ void __launch_bounds__(1024, 1) col_tma16_kernel(const PassParams p, 
         group_sync(1 + g, GT);
 #pragma unroll
         for (int r = 0; r < 32; ++r) v[r] = buf[slot_l + (r << 5)];
+        fence_generic_before_async();              // this thread's stores into the buffer, before the copy engine reuses it
         group_sync(1 + g, GT);                     // the buffer is free: refill it for the tile three ahead
         if (gt == 0 && j + 3 < nitems) issue(j + 3);
         butterflies32<15>(v);                      // row bits 1..4 (register bit 4 = row bit 5 is done)
@@ -386,6 +402,16 @@ __global__ void __launch_bounds__(1024, 1) col_tma16_kernel(const PassParams p, 
         const uint32_t i_l = i_tile + ((w << 6) | h) * step + c;
 #pragma unroll
         for (int r = 0; r < 32; ++r) __stcg(dst + i_l + (r << 1) * step, v[r]);
+    }
+    // Both groups meet here, whether they finished or gave up.  In a healthy run every issued copy has
+    // been taken; after a timeout the copies still in flight get one more bounded wait, so that the
+    // engine is not left writing into shared memory that the next block of this SM may own.
+    __syncthreads();
+    if (tid == 0) {
+        for (int b = 0; b < 3; ++b) {
+            if (s_issued[b] > s_taken[b]) mbar_wait(full + b, (uint32_t)((s_issued[b] - 1) & 1));
+            mbar_inval(full + b);
+        }
     }
 }
 

@@ -176,6 +176,25 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
     return false;
 }
 
+__device__ __forceinline__ void mbar_inval(uint64_t* bar)
+{
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Every thread that touched a shared-memory buffer through ordinary loads and stores runs this
+// before the barrier after which one thread hands the buffer to the asynchronous copy engine.
+__device__ __forceinline__ void fence_generic_before_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// ---- shared by the translation units of the C-ABI (not exported) -----------------------------
+// thread-local last CUDA error behind fosgd_last_cuda_error()
+__attribute__((visibility("hidden"))) void set_last_cuda_error(int e);
+// argument checks of fosgd_decode without the scratch: FOSGD_OK, FOSGD_EINVAL, FOSGD_EALIGN or FOSGD_EUNSUPPORTED
+__attribute__((visibility("hidden"))) int check_decode_args(const void* bits, int64_t d, float lambda, int block_log2,
+                                                            const void* out);
+
 // ---- host-visible launchers (one translation unit per family) --------------------------
 cudaError_t launch_row(int T, int src, int sink, const PassParams& p, cudaStream_t s);
 cudaError_t launch_col(int A, int src, const PassParams& p, cudaStream_t s);

@@ -12,6 +12,7 @@
 #include <cuda_runtime.h>
 
 #include "../../include/fosgd.h"
+#include "common.cuh"
 
 namespace {
 
@@ -49,14 +50,20 @@ extern "C" int fosgd_decode_noalloc(const uint32_t* bits, int64_t d, uint32_t wo
                                     uint64_t step, float lambda, int block_log2, float* out,
                                     fosgd_stream stream)
 {
+    // the decoder's own argument checks come first, so that a bad pointer reads as such at any size
+    int st = fosgd::check_decode_args(bits, d, lambda, block_log2, out);
+    if (st != FOSGD_OK) return st;
     size_t need = 0;
-    int st = fosgd_workspace_bytes(FOSGD_OP_DECODE, d, 1, FOSGD_F32, block_log2, 1, &need);
+    st = fosgd_workspace_bytes(FOSGD_OP_DECODE, d, 1, FOSGD_F32, block_log2, 1, &need);
     if (st != FOSGD_OK) return st;
     if (need > kScratchBytes) return FOSGD_ELIMIT;
     void* ptr = nullptr;
     if (need > 0) {
         const cudaError_t e = scratch_address(&ptr);
-        if (e != cudaSuccess) return FOSGD_ECUDA;
+        if (e != cudaSuccess) {
+            fosgd::set_last_cuda_error((int)e);
+            return FOSGD_ECUDA;
+        }
     }
     // The decoder overwrites every scratch entry it later reads, so nothing has to be cleared
     // between calls even though the array keeps what the previous call left in it.

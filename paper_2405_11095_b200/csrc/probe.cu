@@ -1,0 +1,81 @@
+// Issue-rate probe (measurement aid; the paper has no counterpart).  One kernel per instruction
+// kind keeps every SM's four schedulers busy with independent dependency chains held in
+// registers, so that lane operations per second = (threads x iterations x operations per
+// iteration) / elapsed time is the rate the plain ALUs sustain for that kind on this device at
+// the clock it actually runs.  The benchmark divides the path's algorithmic operation count by
+// this figure instead of by a data-sheet number.
+#include <cuda_runtime.h>
+
+#include "../../include/fosgd.h"
+#include "common.cuh"
+
+namespace fosgd {
+namespace {
+
+constexpr int kChains = 8;    // independent chains per thread (latency is hidden by 64 warps x 8)
+constexpr int kUnroll = 16;   // applications per chain and loop iteration
+constexpr int kThreads = 256;
+constexpr int kBlocksPerSm = 8;
+
+template <int KIND>
+__global__ void __launch_bounds__(kThreads) issue_probe_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink)
+{
+    uint32_t x[kChains];
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) x[c] = (threadIdx.x + 1u) * (2u * c + 1u) + blockIdx.x;
+    const float fa = __uint_as_float(0x33800000u | (a & 0xFFFFu));   // a small positive increment
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                if (KIND == FOSGD_PROBE_FADD) {
+                    x[c] = __float_as_uint(__uint_as_float(x[c]) + fa);
+                } else if (KIND == FOSGD_PROBE_FFMA) {
+                    x[c] = __float_as_uint(fmaf(__uint_as_float(x[c]), 0.999f, fa));
+                } else if (KIND == FOSGD_PROBE_LOP3) {
+                    x[c] = (x[c] ^ x[(c + 1) % kChains]) & (a | x[(c + 3) % kChains]);   // one three-input logic op per step, chains entangled
+                } else {
+                    x[c] = x[c] * a + b;                                               // 32-bit multiply-add
+                }
+            }
+        }
+    }
+    uint32_t s = 0;
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) s ^= x[c];
+    if (s == 0x9E3779B9u && iters < 0) sink[0] = s;   // never true: keeps the chains alive
+}
+
+template <int KIND>
+cudaError_t launch_probe(int blocks, int iters, uint32_t* sink, cudaStream_t s)
+{
+    issue_probe_kernel<KIND><<<blocks, kThreads, 0, s>>>(iters, 0x00012345u, 0x9E3779B9u, sink);
+    return cudaGetLastError();
+}
+
+}  // namespace
+}  // namespace fosgd
+
+using namespace fosgd;
+
+extern "C" int fosgd_probe_issue_rate(int kind, int iters, double* lane_ops, uint32_t* sink, fosgd_stream stream)
+{
+    if (lane_ops == nullptr || sink == nullptr || iters < 1 || iters > (1 << 24)) return FOSGD_EINVAL;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) { set_last_cuda_error((int)e); return FOSGD_ECUDA; }
+    const int blocks = sms * kBlocksPerSm;
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (kind) {
+        case FOSGD_PROBE_FADD: e = launch_probe<FOSGD_PROBE_FADD>(blocks, iters, sink, s); break;
+        case FOSGD_PROBE_FFMA: e = launch_probe<FOSGD_PROBE_FFMA>(blocks, iters, sink, s); break;
+        case FOSGD_PROBE_LOP3: e = launch_probe<FOSGD_PROBE_LOP3>(blocks, iters, sink, s); break;
+        case FOSGD_PROBE_IMAD: e = launch_probe<FOSGD_PROBE_IMAD>(blocks, iters, sink, s); break;
+        default: return FOSGD_EINVAL;
+    }
+    if (e != cudaSuccess) { set_last_cuda_error((int)e); return FOSGD_ECUDA; }
+    *lane_ops = (double)blocks * kThreads * (double)iters * kChains * kUnroll;
+    return FOSGD_OK;
+}

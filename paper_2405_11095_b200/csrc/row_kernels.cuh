@@ -416,7 +416,14 @@ __global__ void __launch_bounds__(1 << (T - 5), min_blocks<T, SINK>()) row_strea
 
         // bounded wait; the block then agrees on the outcome, so that it stops as a whole
         if (!__syncthreads_and(mbar_wait(bar, parity) ? 1 : 0)) {
-            if (tid == 0) atomicAdd(&g_async_wait_timeouts, 1);
+            // the one copy in flight is the one that did not arrive: a second bounded wait, so that the
+            // engine is not left writing into shared memory that the next block of this SM may own
+            if (tid == 0) {
+                atomicAdd(&g_async_wait_timeouts, 1);
+                mbar_wait(bar, parity);
+                mbar_inval(bar);
+            }
+            __syncthreads();
             return;
         }
         parity ^= 1u;
@@ -438,6 +445,7 @@ __global__ void __launch_bounds__(1 << (T - 5), min_blocks<T, SINK>()) row_strea
         }
         butterflies32<31>(v);
         store_round_F<T>(smem, baseF, v);
+        fence_generic_before_async();   // (the landing buffer is only read by the threads, never written)
         __syncthreads();   // round F complete: the landing buffer is free, nobody is in the previous item
         if (tid == 0 && j + 1 < nitems) bulk_load(landing, item_src(j + 1), kTileBytes, bar);
         if (kFinal && tid < C::FLIP_WORDS / 4) {

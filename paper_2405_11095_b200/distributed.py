@@ -121,7 +121,11 @@ def _encode_on_streams(codec, grads, d, buf, lam, seed, step, first, block_log2,
         buf.side_streams = [torch.cuda.Stream() for _ in range(nstreams)]
     cur = torch.cuda.current_stream()
     per = -(-rows // nstreams)
-    ws_per = buf.ws.numel() // rows if buf.ws is not None else 0
+    ws_per = (buf.ws.numel() // rows) & ~15 if buf.ws is not None else 0    # slices stay 16-byte aligned
+    need = codec.workspace_bytes(codec.OP_ENCODE, d, block_log2=block_log2)
+    if ws_per < need:
+        raise ValueError(f"encode_streams needs scratch for every resident row: {need} bytes per row, "
+                         f"{ws_per} available")
     for k, s in enumerate(buf.side_streams):
         a, b = k * per, min(rows, (k + 1) * per)
         if a >= b:

@@ -87,7 +87,7 @@ class OracleCodec:
         cls.downlink_decode(down, d, out, cls._amp(lam_s, per_block), seed, step, **kw)
 
     # ---- what closed_loop.run needs besides the calls above ----
-    OP_AGGREGATE, OP_AMPLITUDES, OP_BLOCK_AMPLITUDES = 2, 5, 6
+    OP_ENCODE, OP_AGGREGATE, OP_AMPLITUDES, OP_BLOCK_AMPLITUDES = 0, 2, 5, 6
     padded_dim = staticmethod(oracle.padded_dim)
     planes = staticmethod(oracle.planes)
 

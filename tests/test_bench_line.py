@@ -40,6 +40,12 @@ def test_gpu_arm_line():
     r = line["roofline"]
     assert {"bound", "achieved", "peak", "unit", "frac", "traffic"} <= set(r)
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    # the fraction is on the method's own bytes; the kernel's own traffic (intermediates included) is listed apart
+    assert r["algorithmic_bytes_per_launch"] <= r["implementation_bytes_per_launch"]
+    assert r["frac"] <= r["implementation_frac"] + 1e-12 and r["call"]["frac"] <= r["implementation_frac"]
+    assert set(r["per_kernel"]) == set(line["kernels"])
+    assert line["repeats"] >= 1 and line["clocks"]["samples"] >= 10
+    assert line["path_roofline"]["alu_peak_source"].startswith("measured") and line["alu_probe"]["lane_ops_per_s"]["fadd"] > 1e13
     e = line["e2e"]
     assert e["h2d_bytes_per_step"] == 16 * (1 << 20) * 4 and e["d2h_bytes_per_step"] == (1 << 20) * 4
     assert 0 < e["value"] < line["value"]

@@ -31,11 +31,16 @@ def test_noalloc_decoder_matches_decoder_twice():
         F.decode(bits, d, ref, lam, seed, step, wid, ws=ws)
         out = torch.full((d,), float("nan"), dtype=torch.float32, device="cuda")
         torch.cuda.synchronize()
-        before = torch.cuda.memory_allocated()
+        # free device memory as the driver reports it (this sees a cudaMalloc made by anyone in the
+        # process, which torch's own counters would not); the first call on a device may still load
+        # the library's kernels, so the comparison starts with the second
+        before = (torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0])
         status = lib.fosgd_decode_noalloc(bits.data_ptr(), d, wid, seed, step, lam, 0, out.data_ptr(), stream)
         assert status == F.OK
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.memory_allocated() == before[0]
+        if call > 0:
+            assert torch.cuda.mem_get_info()[0] == before[1]
         err = (out.double() - ref.double()).norm() / ref.double().norm()
         assert float(err) <= L2_RTOL
         assert torch.equal(out, ref)      # same kernels, same order: bit identical
@@ -52,3 +57,16 @@ def test_noalloc_decoder_rejects_oversize():
     assert e.value.status == F.ELIMIT
     assert "2^20" in str(e.value)
     assert not out.any()                   # nothing was enqueued
+    # the decoder's own argument checks come before the size limit
+    lib = F.lib()
+    stream = torch.cuda.current_stream().cuda_stream
+    assert lib.fosgd_decode_noalloc(0, d, 3, 1, 2, 0.5, 0, out.data_ptr(), stream) == F.EINVAL
+    assert lib.fosgd_decode_noalloc(bits.data_ptr(), d, 3, 1, 2, -1.0, 0, out.data_ptr(), stream) == F.EINVAL
+    assert lib.fosgd_decode_noalloc(bits.data_ptr() + 4, d, 3, 1, 2, 0.5, 0, out.data_ptr(), stream) == F.EALIGN
+    # blocks of 2^15 are single-pass transforms: no scratch, so no limit on d'
+    bits15 = torch.zeros(F.padded_dim(d, 15) // 32, dtype=torch.int32, device="cuda")
+    ref = torch.empty(d, dtype=torch.float32, device="cuda")
+    F.decode(bits15, d, ref, 0.5, 1, 2, 3, block_log2=15)
+    F.decode_noalloc(bits15, d, out, 0.5, 1, 2, 3, block_log2=15)
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref)
