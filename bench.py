@@ -244,7 +244,7 @@ def run_reference(args):
 def label_parts(label):
     name, workers = label.split("@")
     src, sink = name.split(":")[1].split("->")
-    return src, sink, int(workers)
+    return src, sink, 1 if workers == "srv" else int(workers)
 
 
 def implementation_bytes(label, dp, P):
@@ -453,7 +453,7 @@ def analyse(rec, peaks, peak_kind, alu_peak, alu_peak_kind, world):
     def call_ms(pred):
         return sum(v["ms_per_step"] for k, v in kernels.items() if pred(k))
 
-    many = (lambda k: not k.endswith("@1")) if R > 1 else (lambda k: False)
+    many = lambda k: not k.endswith("@srv")      # the workers' kernels; "@srv" marks the server's own vector
     up_ms = call_ms(lambda k: is_uplink_kernel(k) and many(k))
     agg_ms = call_ms(lambda k: not is_uplink_kernel(k) and many(k))
     dn_enc_ms = call_ms(lambda k: is_uplink_kernel(k) and "norm" not in k and not many(k))
@@ -470,10 +470,9 @@ def analyse(rec, peaks, peak_kind, alu_peak, alu_peak_kind, world):
     path("uplink_encode", up_ms, M * (d * esize + dp / 8), {"elems_per_s": M * d / up_ms * 1e3 if up_ms else None})
     path("server_decode_average", agg_ms, M * dp / 8 + 4 * dp + 8 * dp * (chunks - 1),
          {"elems_per_s": M * d / agg_ms * 1e3 if agg_ms else None})
-    if R > 1:
-        path("server_downlink_encode", dn_enc_ms, 4 * dp + P * dp / 8)
-        # every worker computes the same vector: one decode is timed, M of them would run in a deployment
-        path("worker_downlink_decode", dn_dec_ms, P * dp / 8 + 4 * d, {"ms_times_workers": dn_dec_ms * M * world})
+    path("server_downlink_encode", dn_enc_ms, 4 * dp + P * dp / 8)
+    # every worker computes the same vector: one decode is timed, M of them would run in a deployment
+    path("worker_downlink_decode", dn_dec_ms, P * dp / 8 + 4 * d, {"ms_times_workers": dn_dec_ms * M * world})
 
     per_kernel = {}
     for lab, v in kernels.items():

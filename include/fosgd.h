@@ -226,7 +226,18 @@ int fosgd_async_timeouts(int* count);
  * kernel's duration.  Setting the array resets the launch counter.  Thread local. */
 int fosgd_trace_passes(void** events, int capacity);
 int fosgd_trace_count(void);            /* launches recorded since the array was set */
-const char* fosgd_trace_label(int k);   /* e.g. "col10:f32->ws@32", "row14:ws->pack1@32" (kernel, source->sink, workers); valid until the next call */
+const char* fosgd_trace_label(int k);   /* e.g. "col10:f32->ws@4", "row14:ws->pack1@4", "row14:ws16->final@srv" (kernel, source->sink,
+                                           workers of the launch, or "srv" for the server's own vector on the downlink); valid until the next call */
+
+/* Kernel choice for the ten strided stages of a decoder that starts from one packed plane (transform
+ * lengths 2^20 .. 2^25: fosgd_decode, fosgd_server_aggregate, and the downlink decoder with K = 1).
+ * The recursion H_k = H_1 (x) H_{k-1} below Def. 3.4 makes H_1024 = H_8 (x) H_128 a legal factor; with
+ * on != 0 those stages run as H_8 on packed bytes plus a 128 x 128 x 128 8-bit integer product per
+ * block on the tensor cores (tcgen05, accumulators in tensor memory), otherwise in packed fp16
+ * arithmetic on the plain ALUs.  Both give the same fp16 intermediate bit for bit (the values are
+ * integers of magnitude <= 1024).  Default 0: measured on a B200, the plain-ALU kernel is the faster
+ * of the two.  Process-wide; returns the previous setting. */
+int fosgd_set_tensor_core_pass(int on);
 
 /* Issue-rate probe (measurement aid; no counterpart in the paper).  Enqueues one kernel that
  * keeps every scheduler of every SM busy with independent register-resident chains of one

@@ -26,7 +26,7 @@ EXPORTS = ("fosgd_padded_dim", "fosgd_planes", "fosgd_lambda", "fosgd_lambda_ser
            "fosgd_last_cuda_error", "fosgd_version", "fosgd_trace_passes", "fosgd_trace_count",
            "fosgd_trace_label", "fosgd_decode_noalloc", "fosgd_async_timeouts", "fosgd_amplitudes",
            "fosgd_encode_dev", "fosgd_server_aggregate_dev", "fosgd_downlink_decode_dev", "fosgd_downlink_apply",
-           "fosgd_downlink_encode", "fosgd_probe_issue_rate")
+           "fosgd_downlink_encode", "fosgd_probe_issue_rate", "fosgd_set_tensor_core_pass")
 
 
 class FosgdError(RuntimeError):
@@ -67,6 +67,7 @@ def _load() -> C.CDLL:
     L.fosgd_downlink_apply.argtypes = [vp, i64, u64, u64, C.c_float, vp, cint, cint, cint, C.c_float, vp, vp, sz, vp]
     L.fosgd_downlink_decode_dev.argtypes = [vp, i64, u64, u64, vp, cint, cint, cint, vp, vp, sz, vp]
     L.fosgd_probe_issue_rate.argtypes = [cint, cint, C.POINTER(dbl), vp, vp]
+    L.fosgd_set_tensor_core_pass.argtypes, L.fosgd_set_tensor_core_pass.restype = [cint], cint
     L.fosgd_strerror.argtypes, L.fosgd_strerror.restype = [cint], C.c_char_p
     L.fosgd_last_cuda_error.restype = cint
     L.fosgd_version.restype = C.c_char_p
@@ -262,6 +263,12 @@ def downlink_apply(down_bits, d, x, lam_s, seed, step, step_size, K=1, block_log
                                      _ptr(dev), int(per_block), K, block_log2, float(step_size), _ptr(x),
                                      _ptr(ws), _nbytes(ws), _stream()), "fosgd_downlink_apply")
     return x
+
+
+def set_tensor_core_pass(on: bool) -> bool:
+    """fosgd_set_tensor_core_pass: run the strided decode pass from packed bits on the tensor cores
+    (True) or on the plain ALUs (False, the default and the faster one); returns the previous setting."""
+    return bool(_lib.fosgd_set_tensor_core_pass(int(bool(on))))
 
 
 PROBE_FADD, PROBE_FFMA, PROBE_LOP3, PROBE_IMAD = range(4)

@@ -26,7 +26,7 @@ def _nvcc() -> str:
 def _units():
     units = [("api.cu", "api.o", []), ("col_kernels.cu", "col_kernels.o", []),
              ("small_kernels.cu", "small_kernels.o", []), ("noalloc.cu", "noalloc.o", []), ("amplitudes.cu", "amplitudes.o", []),
-             ("probe.cu", "probe.o", [])]
+             ("probe.cu", "probe.o", []), ("tc_kernels.cu", "tc_kernels.o", [])]
     units += [("row_inst.cu", f"row_{t}.o", [f"-DFOSGD_ROW_T={t}"]) for t in ROW_TILES]
     return units
 

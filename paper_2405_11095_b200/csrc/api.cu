@@ -3,6 +3,8 @@
 #include <math.h>
 #include <stdio.h>
 
+#include <atomic>
+
 #include "../../include/fosgd.h"
 #include "common.cuh"
 
@@ -41,7 +43,7 @@ thread_local int g_last_cuda_error = 0;
 
 // Optional per-launch timing hooks (fosgd_trace_passes): caller-owned events, recorded around
 // every kernel launch issued by this thread.
-struct TraceEntry { char kind; int size, src, sink, workers; };
+struct TraceEntry { char kind; int size, src, sink, workers; };   // workers = 0: the server's own vector (downlink)
 thread_local cudaEvent_t* g_trace_events = nullptr;
 thread_local int g_trace_capacity = 0;
 thread_local int g_trace_count = 0;
@@ -55,10 +57,11 @@ cudaError_t traced(char kind, int size, int src, int sink, const PassParams& p, 
     cudaError_t e = kind == 'r' ? launch_row(size, src, sink, p, s)
                   : kind == 'c' ? launch_col(size, src, p, s)
                   : kind == 'h' ? launch_colh(size, p, s)
+                  : kind == 't' ? launch_tc_col(p, s)
                                 : launch_small(size, src, sink, p, s);
     if (on) {
         cudaEventRecord(g_trace_events[2 * g_trace_count + 1], s);
-        g_trace_log[g_trace_count] = TraceEntry{kind, size, src, sink, p.nworkers};
+        g_trace_log[g_trace_count] = TraceEntry{kind, size, src, sink, p.id0 == FOSGD_SERVER_ID ? 0 : p.nworkers};
         ++g_trace_count;
     }
     return e;
@@ -163,6 +166,11 @@ Rng make_rng(uint64_t seed, uint64_t step)
     return r;
 }
 
+// which kernel runs the ten strided stages of a decoder whose source is one packed plane: 0 = packed
+// fp16 arithmetic on the plain ALUs (the faster one as measured, hence the default), 1 = tensor cores
+std::atomic<int> g_tensor_core_pass{0};
+bool tc_enabled() { return g_tensor_core_pass.load(std::memory_order_relaxed) != 0; }
+
 // Enqueue one source -> sink transform for p.nworkers workers.  Workers are processed in
 // chunks of as many as the scratch buffer holds; SINK_FINAL accumulates chunk after chunk.
 int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, size_t ws_bytes,
@@ -170,13 +178,13 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
 {
     const Plan& pl = g.plan;
     cudaError_t e = cudaSuccess;
+#define FOSGD_CUDA_OK(call) do { e = (call); if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; } } while (0)
     if (pl.ncol == 0) {
-        e = (pl.L < 10) ? traced('s', pl.L, src, sink, p, s) : traced('r', pl.T, src, sink, p, s);
-        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
+        FOSGD_CUDA_OK((pl.L < 10) ? traced('s', pl.L, src, sink, p, s) : traced('r', pl.T, src, sink, p, s));
         return FOSGD_OK;
     }
     if (ws == nullptr || ws_bytes < g.ws_per_worker) return FOSGD_EWORKSPACE;
-    size_t cap = ws_bytes / g.ws_per_worker;
+    const size_t cap = ws_bytes / g.ws_per_worker;
     const int total = p.nworkers;
     const int chunk = (int)(cap < (size_t)total ? cap : (size_t)total);
     const float final_scale = p.scale;
@@ -192,39 +200,30 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
         q.nworkers = m;
         q.id0 = id0 + (uint32_t)n0;
         if (p.amp_dev) q.amp_dev = p.amp_dev + (int64_t)n0 * p.amp_stride;
+        const void* const srck = src0 + (size_t)n0 * (size_t)p.src_stride * src_elem_bytes(src);
+        bool tensor_pass = false;
         if (half_path) {
             PassParams pc = q;
-            pc.src = src0 + (size_t)n0 * (size_t)p.src_stride * src_elem_bytes(src);
+            pc.src = srck;
             pc.dst = ws;
             pc.dst_stride = g.dp;
             pc.lo_log = pl.lo[0];
-            e = traced('h', pl.A[0], SRC_BITS, 4, pc, s);
-            if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
-            PassParams pr = q;
-            pr.src = ws;
-            pr.src_stride = g.dp;
-            if (sink == SINK_FINAL) {
-                pr.overwrite = (n0 == 0) ? first_overwrite : 0;
-                pr.scale = (n0 + m == total) ? final_scale : 1.f;
-                if (p.amp_mode == AMP_SCALE && n0 + m != total) pr.amp_mode = AMP_DITHER;
-            } else {
-                pr.dst = dst0 + (size_t)n0 * (size_t)p.dst_stride * sink_elem_bytes(sink);
+            // ten stages: H_8 on packed bytes + H_128 on the tensor cores, same fp16 intermediate
+            tensor_pass = pl.A[0] == 10 && tc_enabled() && tc_col_applicable(pc);
+            if (tensor_pass) FOSGD_CUDA_OK(traced('t', pl.A[0], SRC_BITS, 4, pc, s));
+            else FOSGD_CUDA_OK(traced('h', pl.A[0], SRC_BITS, 4, pc, s));
+        } else {
+            // strided passes, highest bits first: source -> ws, then ws -> ws in place
+            for (int c = pl.ncol - 1; c >= 0; --c) {
+                PassParams pc = q;
+                const bool first = (c == pl.ncol - 1);
+                pc.src = first ? srck : ws;
+                pc.src_stride = first ? p.src_stride : g.dp;
+                pc.dst = ws;
+                pc.dst_stride = g.dp;
+                pc.lo_log = pl.lo[c];
+                FOSGD_CUDA_OK(traced('c', pl.A[c], first ? src : (int)SRC_WS, SINK_WS, pc, s));
             }
-            e = traced('r', pl.T, SRC_WS16, sink, pr, s);
-            if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
-            continue;
-        }
-        // strided passes, highest bits first: source -> ws, then ws -> ws in place
-        for (int c = pl.ncol - 1; c >= 0; --c) {
-            PassParams pc = q;
-            const bool first = (c == pl.ncol - 1);
-            pc.src = first ? static_cast<const void*>(src0 + (size_t)n0 * (size_t)p.src_stride * src_elem_bytes(src)) : ws;
-            pc.src_stride = first ? p.src_stride : g.dp;
-            pc.dst = ws;
-            pc.dst_stride = g.dp;
-            pc.lo_log = pl.lo[c];
-            e = traced('c', pl.A[c], first ? src : (int)SRC_WS, SINK_WS, pc, s);
-            if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
         }
         PassParams pr = q;
         pr.src = ws;
@@ -236,9 +235,9 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
         } else {
             pr.dst = dst0 + (size_t)n0 * (size_t)p.dst_stride * sink_elem_bytes(sink);
         }
-        e = traced('r', pl.T, SRC_WS, sink, pr, s);
-        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
+        FOSGD_CUDA_OK(traced('r', pl.T, half_path ? (int)SRC_WS16 : (int)SRC_WS, sink, pr, s));
     }
+#undef FOSGD_CUDA_OK
     return FOSGD_OK;
 }
 
@@ -604,8 +603,11 @@ int fosgd_async_timeouts(int* count)
                                         row_timeouts_13, row_timeouts_14, row_timeouts_15};
     int total = 0;
     {
-        const cudaError_t e = col_timeouts(&total);
+        int t = 0;
+        cudaError_t e = col_timeouts(&total);
+        if (e == cudaSuccess) e = tc_timeouts(&t);
         if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
+        total += t;
     }
     for (auto fn : fns) {
         int c = 0;
@@ -634,10 +636,18 @@ const char* fosgd_trace_label(int k)
     static const char* const srcs[] = {"f32", "bf16", "bits", "ws", "ws16"};
     static const char* const sinks[] = {"ws", "pack1", "packK", "final", "ws16", "amp"};
     const TraceEntry& t = g_trace_log[k];
-    snprintf(g_trace_label, sizeof g_trace_label, "%s%d:%s->%s@%d",
-             t.kind == 'r' ? "row" : (t.kind == 'c' ? "col" : (t.kind == 'h' ? "colh" : (t.kind == 'n' ? "norm" : "small"))), t.size, srcs[t.src], sinks[t.sink],
-             t.workers);
+    char who[16];
+    if (t.workers > 0) snprintf(who, sizeof who, "%d", t.workers);
+    else snprintf(who, sizeof who, "srv");
+    snprintf(g_trace_label, sizeof g_trace_label, "%s%d:%s->%s@%s",
+             t.kind == 'r' ? "row" : (t.kind == 'c' ? "col" : (t.kind == 'h' ? "colh" : (t.kind == 'n' ? "norm" : (t.kind == 't' ? "tc" : "small")))), t.size, srcs[t.src], sinks[t.sink],
+             who);
     return g_trace_label;
+}
+
+int fosgd_set_tensor_core_pass(int on)
+{
+    return g_tensor_core_pass.exchange(on ? 1 : 0, std::memory_order_relaxed);
 }
 
 const char* fosgd_version(void) { return "libfosgd 0.1 (sm_100a)"; }

@@ -11,6 +11,7 @@
 //           after one exchange through shared memory.
 #include <cuda.h>   // CUtensorMap and the encode entry point type; the driver is reached through the runtime
 
+#include "col4.cuh"
 #include "common.cuh"
 
 namespace fosgd {
@@ -234,191 +235,28 @@ __global__ void __launch_bounds__(1 << (A - 1), 2) col_tile16_kernel(const PassP
     for (int r = 0; r < 32; ++r) __stcg(dst + i_l + r * step, v[r]);   // L2 only: read next by another kernel
 }
 
-// ---- A = 10, fp32 sources, TMA-staged persistent pipeline ------------------------------------------
-// The 16-column tile once more, with the tile fetched by the tensor copy engine.  The source is
-// described by a 3-D tensor map (columns S, rows, workers); a tile is four box copies of 256 rows x
-// 16 columns landing densely in a 64 KiB buffer and completing on one mbarrier.  Rows past the end
-// of the gradient are zero-filled by the copy engine (the map only covers whole rows; a last,
-// partial row is patched in by ordinary loads).  A dense buffer admits no padding, so both rounds
-// keep row bit 0 in the lane (a warp always touches two adjacent rows = 32 consecutive words) and
-// the butterfly on row bit 0 is one shuffle stage: round F transforms row bits 5..9, round L bits
-// 1..4, the shuffle bit 0.  Blocks are persistent: two groups of 512 threads take tiles in turn over
-// three buffers, and the group that has pulled its tile into registers for round L starts the
-// copies of the tile three positions ahead into the buffer it has just freed, so loads stay in
-// flight while both groups compute and store.
+// ---- A = 10, gradients or the fp32 intermediate: tiles staged by the tensor copy engine (col4.cuh) ----
 static __device__ int g_col_wait_timeouts;   // groups that abandoned a bounded wait
 
-// bar.sync / bar.red are the warp-aligned forms: every lane of a warp must arrive together.  The
-// code before them has lane-dependent paths (one lane issues the copies, sixteen patch a row, the
-// polling loop of a bounded wait ends per lane), and nothing obliges the compiler to have rejoined
-// them in front of an opaque asm statement, so the warp is converged explicitly first.
-__device__ __forceinline__ void group_sync(int id, int nthreads)
+__global__ void __launch_bounds__(512, 2) col4_kernel(const PassParams p, const __grid_constant__ CUtensorMap tmap,
+                                                      const int nruns, const uint32_t full_rows)
 {
-    __syncwarp();
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    col4_run(p, &tmap, full_rows, (int)(blockIdx.x / (unsigned)nruns), (blockIdx.x % (unsigned)nruns) * 8u, smem_raw,
+             (int)threadIdx.x, &g_col_wait_timeouts);
 }
 
-// barrier + AND over the group: every thread learns whether all of them saw `ok`
-__device__ __forceinline__ bool group_all(int id, int nthreads, bool ok)
+__global__ void __launch_bounds__(1024, 1) col4_duo_kernel(const PassParams p, const __grid_constant__ CUtensorMap tmap,
+                                                           const int nruns, const uint32_t full_rows)
 {
-    uint32_t all;
-    __syncwarp();
-    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, %2, %3, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
-                 : "=r"(all) : "r"((uint32_t)ok), "r"(id), "r"(nthreads) : "memory");
-    return all != 0;
-}
-
-template <int SRC>
-__global__ void __launch_bounds__(1024, 1) col_tma16_kernel(const PassParams p, const __grid_constant__ CUtensorMap tmap,
-                                                            const int64_t nsegs, const uint32_t full_rows)
-{
-    static_assert(SRC == SRC_G32 || SRC == SRC_WS, "4-byte elements only");
-    constexpr int A = 10;
-    constexpr int GT = 512;                                 // threads per group
-    constexpr int BUF_WORDS = (1 << A) * 16;
-    extern __shared__ __align__(128) float smem[];
-    uint64_t* const full = reinterpret_cast<uint64_t*>(smem + 3 * BUF_WORDS);
-    // Copies issued into / tiles taken out of each buffer (written by one thread of the issuing resp.
-    // consuming group), and the flag that stops all issuing once a bounded wait has given up: the
-    // block then drains what is still in flight before any of its threads exits.
-    __shared__ int s_issued[3], s_taken[3], s_stop;
-
-    const int tid = threadIdx.x;
-    const int g = tid >> 9;
-    const int gt = tid & (GT - 1);
-    const uint32_t lane = gt & 31, c = lane & 15, h = lane >> 4, w = gt >> 5;
-    const uint32_t step = 1u << p.lo_log;
-    const uint32_t d32 = (uint32_t)p.d;
-    const int64_t total = nsegs * p.nworkers;
-    const int64_t nitems = (total - (int64_t)blockIdx.x + gridDim.x - 1) / gridDim.x;
-
-    if (tid == 0) {
-        for (int b = 0; b < 3; ++b) {
-            mbar_init(full + b, 1);
-            s_issued[b] = 0;
-            s_taken[b] = 0;
-        }
-        s_stop = 0;
-    }
-    __syncthreads();
-
-    auto item_coords = [&](int64_t j, int& n, uint32_t& lo0, uint32_t& hi) {
-        const int64_t q = blockIdx.x + j * gridDim.x;
-        n = (int)(q / nsegs);
-        const int64_t seg = q % nsegs;
-        lo0 = (uint32_t)((seg << 4) & (((int64_t)1 << p.lo_log) - 1));
-        hi = (uint32_t)((seg << 4) >> p.lo_log);
-    };
-    // one thread: four box copies (256 rows x 16 columns each) into buffer j % 3
-    auto issue = [&](int64_t j) {
-        if (*(volatile int*)&s_stop) return;
-        int n;
-        uint32_t lo0, hi;
-        item_coords(j, n, lo0, hi);
-        uint64_t* const bar = full + (j % 3);
-        const uint32_t dst0 = smem_u32(smem + (j % 3) * BUF_WORDS);
-        s_issued[j % 3] += 1;
-        fence_generic_before_async();
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(65536u) : "memory");
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                         ::"r"(dst0 + 16384u * q), "l"(&tmap), "r"((int)lo0), "r"((int)((hi << A) + 256 * q)),
-                           "r"(n), "r"(smem_u32(bar)) : "memory");
-        }
-    };
-
-    if (gt == 0) {
-        if (g == 0) {
-            if (nitems > 0) issue(0);
-            if (nitems > 2) issue(2);
-        } else {
-            if (nitems > 1) issue(1);
-        }
-    }
-
-    const int slot_f = (int)((w << 5) | (h << 4) | c);     // round F: row = (r << 5) | (w << 1) | h, + (r << 9)
-    const int slot_l = (int)((w << 10) | (h << 4) | c);    // round L: row = (w << 6) | (r << 1) | h, + (r << 5)
-
-    for (int64_t j = g; j < nitems; j += 2) {
-        float* const buf = smem + (j % 3) * BUF_WORDS;
-        int n;
-        uint32_t lo0, hi;
-        item_coords(j, n, lo0, hi);
-        const uint32_t i_tile = (hi << (p.lo_log + A)) + lo0;
-        const uint32_t bitpos = (lo0 & 31u) + c;
-
-        uint32_t word_lo = 0, word_hi = 0;   // flip words of rows (r = lane & 15, h) and (16 + (lane & 15), h)
-        if (SRC == SRC_G32) {
-            const uint32_t row_a = ((lane & 15u) << 5) | (w << 1) | h;
-            const uint32_t ia = i_tile + row_a * step, ib = ia + (step << 9);
-            word_lo = eps_word(p.rng, p.id0 + (uint32_t)n, ia >> 5);
-            word_hi = eps_word(p.rng, p.id0 + (uint32_t)n, ib >> 5);
-        }
-        // bounded wait; the group then agrees on the outcome, so that it stops as a whole
-        if (!group_all(1 + g, GT, mbar_wait(full + (j % 3), (uint32_t)((j / 3) & 1)))) {
-            if (gt == 0) {
-                atomicAdd(&g_col_wait_timeouts, 1);
-                *(volatile int*)&s_stop = 1;
-            }
-            break;
-        }
-        if (gt == 0) s_taken[j % 3] += 1;
-        if (SRC == SRC_G32) {
-            // the map covers whole rows only: a last partial row of the gradient is patched in
-            const uint32_t row_p = full_rows - (hi << A);                  // tile-local index of that row
-            if (row_p < (1u << A) && gt < 16) {
-                const uint32_t i = full_rows * step + lo0 + (uint32_t)gt;
-                if (i < d32)
-                    buf[(row_p << 4) + gt] = (static_cast<const float*>(p.src) + (int64_t)n * p.src_stride)[i];
-            }
-            if (row_p < (1u << A)) group_sync(1 + g, GT);
-        }
-        float v[32];
-        const uint32_t shamt = 31u - bitpos;
-#pragma unroll
-        for (int r = 0; r < 32; ++r) {
-            float x = buf[slot_f + (r << 9)];
-            if (SRC == SRC_G32) {
-                const uint32_t roww = __shfl_sync(0xFFFFFFFFu, r < 16 ? word_lo : word_hi, r & 15, 16);
-                x = flip_shifted(x, roww, shamt);
-            }
-            v[r] = x;
-        }
-        butterflies32<31>(v);                      // row bits 5..9
-#pragma unroll
-        for (int r = 0; r < 32; ++r) buf[slot_f + (r << 9)] = v[r];
-        group_sync(1 + g, GT);
-#pragma unroll
-        for (int r = 0; r < 32; ++r) v[r] = buf[slot_l + (r << 5)];
-        fence_generic_before_async();              // this thread's stores into the buffer, before the copy engine reuses it
-        group_sync(1 + g, GT);                     // the buffer is free: refill it for the tile three ahead
-        if (gt == 0 && j + 3 < nitems) issue(j + 3);
-        butterflies32<15>(v);                      // row bits 1..4 (register bit 4 = row bit 5 is done)
-        const float sgn = h ? -1.f : 1.f;          // row bit 0 lives in the lane: one shuffle stage
-#pragma unroll
-        for (int r = 0; r < 32; ++r) v[r] = fmaf(sgn, v[r], __shfl_xor_sync(0xFFFFFFFFu, v[r], 16));
-        float* const dst = static_cast<float*>(p.dst) + (int64_t)n * p.dst_stride;
-        const uint32_t i_l = i_tile + ((w << 6) | h) * step + c;
-#pragma unroll
-        for (int r = 0; r < 32; ++r) __stcg(dst + i_l + (r << 1) * step, v[r]);
-    }
-    // Both groups meet here, whether they finished or gave up.  In a healthy run every issued copy has
-    // been taken; after a timeout the copies still in flight get one more bounded wait, so that the
-    // engine is not left writing into shared memory that the next block of this SM may own.
-    __syncthreads();
-    if (tid == 0) {
-        for (int b = 0; b < 3; ++b) {
-            if (s_issued[b] > s_taken[b]) mbar_wait(full + b, (uint32_t)((s_issued[b] - 1) & 1));
-            mbar_inval(full + b);
-        }
-    }
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    col4_duo(p, &tmap, (uint32_t)nruns, full_rows, (uint32_t)nruns * (uint32_t)p.nworkers, smem_raw, &g_col_wait_timeouts);
 }
 
 cudaError_t col_timeouts(int* out) { return cudaMemcpyFromSymbol(out, g_col_wait_timeouts, sizeof(int)); }
 
-// Tensor map over the source of a strided pass: (S columns, rows, workers).  False if the driver
-// entry point is missing or refuses the geometry; the caller then uses the plain kernel.
+// Tensor map over the gradients as the strided pass sees them: (S columns, whole rows, workers).
+// False if the driver entry point is missing or refuses the geometry; the caller then uses the plain kernel.
 static bool make_col_tensor_map(CUtensorMap* map, const void* base, uint64_t S, uint64_t rows, uint64_t workers,
                                 uint64_t worker_stride_elems)
 {
@@ -443,26 +281,35 @@ static bool make_col_tensor_map(CUtensorMap* map, const void* base, uint64_t S, 
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int SRC>
-static cudaError_t launch_col_tma(const PassParams& p, cudaStream_t s, bool* launched)
+// Ten stages on fp32 gradients through the copy engine.  *launched stays false where it does not apply
+// (rows shorter than a run of 128 columns, or the driver refuses the map).
+static cudaError_t launch_col4(const PassParams& p, cudaStream_t s, bool* launched)
 {
     constexpr int A = 10;
     *launched = false;
     const uint64_t S = (uint64_t)1 << p.lo_log;
-    const uint64_t rows = (SRC == SRC_WS) ? (uint64_t)(p.dp >> p.lo_log) : (uint64_t)(p.d >> p.lo_log);   // whole rows
+    const uint64_t rows = (uint64_t)(p.d >> p.lo_log);   // whole rows
+    const int64_t nsegs = (p.dp >> A) / 16;
+    const int64_t nruns = nsegs / 8;
+    if (S < 128 || nsegs % 8 != 0 || nruns * p.nworkers > 0x7FFFFFFF) return cudaSuccess;
     CUtensorMap map;
     if (!make_col_tensor_map(&map, p.src, S, rows, (uint64_t)p.nworkers, (uint64_t)p.src_stride)) return cudaSuccess;
-    auto kern = col_tma16_kernel<SRC>;
-    constexpr size_t smem = (size_t)3 * (1 << A) * 16 * 4 + 32;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    int dev = 0, sms = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    const int64_t nsegs = (p.dp >> A) / 16;
-    int64_t blocks = sms;
-    if (blocks > nsegs * p.nworkers) blocks = nsegs * p.nworkers;
-    kern<<<(unsigned)blocks, 1024, smem, s>>>(p, map, nsegs, (uint32_t)rows);
+    cudaError_t e;
+    if (p.lo_log >= 15) {
+        // rows 128 KiB apart or more: the two-group persistent form (0.44 against 0.48 ms on 8 workers of 2^25)
+        if ((e = cudaFuncSetAttribute(col4_duo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Col4Duo::SMEM_BYTES)) != cudaSuccess) return e;
+        int dev = 0, sms = 0;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        int64_t blocks = nruns * p.nworkers;
+        if (blocks > sms) blocks = sms;
+        col4_duo_kernel<<<(unsigned)blocks, 1024, Col4Duo::SMEM_BYTES, s>>>(p, map, (int)nruns, (uint32_t)rows);
+    } else {
+        // one block per run (0.83 against 0.91 ms on 32 workers of 2^24; blocks that start at different times
+        // keep the memory system evenly loaded)
+        if ((e = cudaFuncSetAttribute(col4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Col4::SMEM_BYTES)) != cudaSuccess) return e;
+        col4_kernel<<<(unsigned)(nruns * p.nworkers), 512, Col4::SMEM_BYTES, s>>>(p, map, (int)nruns, (uint32_t)rows);
+    }
     *launched = true;
     return cudaGetLastError();
 }
@@ -616,17 +463,11 @@ static cudaError_t launch_col_one(const PassParams& p, cudaStream_t s)
         const dim3 grid((unsigned)((p.dp >> A) / 256), (unsigned)p.nworkers);
         col_small_kernel<A, SRC><<<grid, 256, 0, s>>>(p);
     } else if constexpr (A >= 8) {
-        // The TMA-staged kernel is used where it has been validated against the oracle: as the single
-        // strided pass of a transform (lengths 2^24 and 2^25), reading the caller's gradients out of
-        // place.  As the in-place second strided pass of the 2^31 transform a launch failed
-        // (unspecified launch failure) and the cause was not found by inspection, so transforms with
-        // two strided passes keep the plain kernel for both.
+        // ten stages on fp32 gradients: the copy-engine kernels, unless the driver refuses the tensor map
         if constexpr (A == 10 && SRC == SRC_G32) {
-            if (p.dp == ((int64_t)1 << (p.lo_log + A)) && p.src != p.dst) {
-                bool launched = false;
-                const cudaError_t e = launch_col_tma<SRC>(p, s, &launched);
-                if (e != cudaSuccess || launched) return e;
-            }
+            bool launched = false;
+            const cudaError_t e = launch_col4(p, s, &launched);
+            if (e != cudaSuccess || launched) return e;
         }
         auto kern = col_tile16_kernel<A, SRC>;
         constexpr size_t smem = (size_t)phys16((1 << A) * 16) * 4;

@@ -65,10 +65,52 @@ __device__ __forceinline__ float amplitude_at(const PassParams& p, int n, int64_
     return p.amp_dev ? __ldg(p.amp_dev + (int64_t)n * p.amp_stride + (i >> p.amp_shift)) : 1.f;
 }
 
-// ---- Philox4x32-10 (Salmon et al., SC'11), written from the published round function ----
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                               uint32_t k0, uint32_t k1)
+// The parameter block of the kernels with a dither sink: PassParams plus the ten round keys of the
+// generator (Weyl sequence of the key), computed once on the host.  As kernel parameters they sit in
+// the constant bank and feed the round's logic instruction directly, which saves the two additions
+// per round that every call would otherwise repeat (4 % of the one-dither pack pass).  The other
+// kernels keep the plain block: with the table in it the flip + accumulate kernels, which never use
+// it, ran 8 % slower.
+struct PassParamsRK : PassParams {
+    uint32_t rk0[10], rk1[10];
+};
+
+inline PassParamsRK with_round_keys(const PassParams& p)
 {
+    PassParamsRK r;
+    static_cast<PassParams&>(r) = p;
+    for (int i = 0; i < 10; ++i) {
+        r.rk0[i] = p.rng.k0 + (uint32_t)i * 0x9E3779B9u;
+        r.rk1[i] = p.rng.k1 + (uint32_t)i * 0xBB67AE85u;
+    }
+    return r;
+}
+
+// ---- Philox4x32-10 (Salmon et al., SC'11), written from the published round function ----
+// Two forms of the same ten rounds.  rng_words_dither takes the round keys from a table in the
+// parameter bank: for the dither sinks, whose every thread makes eight calls per tile.  rng_words
+// advances the key by addition inside the rounds: for the flip words, which a thread generates once
+// or twice per tile.
+__device__ __forceinline__ uint4 rng_words_dither(const PassParamsRK& p, uint32_t id, uint32_t domain, uint32_t c)
+{
+    uint32_t c0 = c, c1 = domain, c2 = p.rng.step_lo, c3 = id;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ p.rk0[r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ p.rk1[r];
+        c0 = n0;
+        c1 = (uint32_t)p1;
+        c2 = n2;
+        c3 = (uint32_t)p0;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+__device__ __forceinline__ uint4 rng_words(const Rng& g, uint32_t id, uint32_t domain, uint32_t c)
+{
+    uint32_t c0 = c, c1 = domain, c2 = g.step_lo, c3 = id, k0 = g.k0, k1 = g.k1;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
@@ -83,11 +125,6 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
         k1 += 0xBB67AE85u;
     }
     return make_uint4(c0, c1, c2, c3);
-}
-
-__device__ __forceinline__ uint4 rng_words(const Rng& g, uint32_t id, uint32_t domain, uint32_t c)
-{
-    return philox4x32_10(c, domain, g.step_lo, id, g.k0, g.k1);
 }
 
 __device__ __forceinline__ uint32_t pick(const uint4& w, uint32_t j)
@@ -188,6 +225,26 @@ __device__ __forceinline__ void fence_generic_before_async()
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// bar.sync / bar.red are the warp-aligned forms: every lane of a warp must arrive together.  The
+// code before them has lane-dependent paths (one lane issues the copies, sixteen patch a row, the
+// polling loop of a bounded wait ends per lane), and nothing obliges the compiler to have rejoined
+// them in front of an opaque asm statement, so the warp is converged explicitly first.
+__device__ __forceinline__ void group_sync(int id, int nthreads)
+{
+    __syncwarp();
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// barrier + AND over the group: every thread learns whether all of them saw `ok`
+__device__ __forceinline__ bool group_all(int id, int nthreads, bool ok)
+{
+    uint32_t all;
+    __syncwarp();
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, %2, %3, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                 : "=r"(all) : "r"((uint32_t)ok), "r"(id), "r"(nthreads) : "memory");
+    return all != 0;
+}
+
 // ---- shared by the translation units of the C-ABI (not exported) -----------------------------
 // thread-local last CUDA error behind fosgd_last_cuda_error()
 __attribute__((visibility("hidden"))) void set_last_cuda_error(int e);
@@ -199,6 +256,9 @@ __attribute__((visibility("hidden"))) int check_decode_args(const void* bits, in
 cudaError_t launch_row(int T, int src, int sink, const PassParams& p, cudaStream_t s);
 cudaError_t launch_col(int A, int src, const PassParams& p, cudaStream_t s);
 cudaError_t launch_colh(int A, const PassParams& p, cudaStream_t s);   // one-plane bits -> fp16 intermediate
+bool tc_col_applicable(const PassParams& p);                            // ten strided stages from one plane on the tensor cores
+cudaError_t launch_tc_col(const PassParams& p, cudaStream_t s);          // one-plane bits -> fp16 intermediate
+cudaError_t tc_timeouts(int* out);
 cudaError_t col_timeouts(int* out);                                      // synchronising read of the strided unit's counter
 cudaError_t launch_small(int L, int src, int sink, const PassParams& p, cudaStream_t s);
 cudaError_t launch_amplitudes(const void* grads, int bf16, int64_t d, int64_t worker_stride, int M, double alpha,

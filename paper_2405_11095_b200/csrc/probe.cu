@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(kThreads) issue_probe_kernel(int iters, uint32
                 } else if (KIND == FOSGD_PROBE_FFMA) {
                     x[c] = __float_as_uint(fmaf(__uint_as_float(x[c]), 0.999f, fa));
                 } else if (KIND == FOSGD_PROBE_LOP3) {
-                    x[c] = (x[c] ^ x[(c + 1) % kChains]) & (a | x[(c + 3) % kChains]);   // one three-input logic op per step, chains entangled
+                    x[c] = (x[c] & x[(c + 1) % kChains]) ^ a;   // one three-input logic op per step, chains entangled
                 } else {
                     x[c] = x[c] * a + b;                                               // 32-bit multiply-add
                 }

@@ -83,15 +83,26 @@ struct RowCfg {
     static_assert(((FMASK | MMASK | LMASK) & ((1u << T) - 1)) == ((1u << T) - 1), "bits uncovered");
 };
 
-// Registers are capped at 64 per thread (2048 resident threads per SM).  The store and one-dither
+// parameter block of a kernel by its sink: the dither sinks carry the generator's round keys
+template <int SINK> struct KernelParams { using type = PassParams; };
+template <> struct KernelParams<SINK_PACK1> { using type = PassParamsRK; };
+template <> struct KernelParams<SINK_PACKK> { using type = PassParamsRK; };
+template <int SINK>
+inline typename KernelParams<SINK>::type kernel_params(const PassParams& p)
+{
+    if constexpr (SINK == SINK_PACK1 || SINK == SINK_PACKK) return with_round_keys(p);
+    else return p;
+}
+
+// Registers are capped at 64 per thread (2048 resident threads per SM).  The store and dither
 // sinks need no more by themselves.  The flip + accumulate sink holds 32 values and 32 sums per
 // thread and would take ~95: capped, it spills a few words but runs twice the warps, which is
-// worth 5 % on the 2^24 workload.  The K-dither sink (32 counters as well) is left uncapped.
+// worth 5 % on the 2^24 workload.
 // (Three blocks of the one-dither sink at 40 registers were measured slower, 0.96 against 0.80 ms.)
 template <int T, int SINK>
 __host__ __device__ constexpr int min_blocks()
 {
-    return (SINK == SINK_PACKK) ? 1 : (1 << (15 - T));
+    return 1 << (15 - T);
 }
 
 // ---- the three rounds on the padded tile ---------------------------------------------------
@@ -133,7 +144,7 @@ __device__ __forceinline__ void sink_ws(const PassParams& p, int n, int64_t i0, 
 
 // Sign bits are shifted into a per-lane mask (bit r = sign of register r), then the 32 x 32 bit
 // matrix is transposed across the warp so that lane r owns packed word r.
-__device__ __forceinline__ void sink_pack1(const PassParams& p, int n, uint32_t id, int64_t i0, uint32_t lane,
+__device__ __forceinline__ void sink_pack1(const PassParamsRK& p, int n, uint32_t id, int64_t i0, uint32_t lane,
                                            const float (&v)[32], float amp)
 {
     const uint32_t cbase = ((uint32_t)(i0 >> 7) << 5) + lane;
@@ -142,11 +153,13 @@ __device__ __forceinline__ void sink_pack1(const PassParams& p, int n, uint32_t 
     uint32_t neg = 0;
 #pragma unroll
     for (int m = 7; m >= 0; --m) {
-        const uint4 w = rng_words(p.rng, id, 1u, cbase + 32u * m);
+        const uint4 w = rng_words_dither(p, id, 1u, cbase + 32u * m);
         const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int q = 3; q >= 0; --q) {
-            // z = (2 k24 + 1 - 2^24) c + y, k24 = top 24 bits of the word
+            // z = (2 k24 + 1 - 2^24) c + y, k24 = top 24 bits of the word (two roundings: the two operations
+            // are independent of each other's latency, 4 % faster than the single-rounding form of the
+            // K-dither sink, and with one dither per coordinate the ties stay far inside the allowance)
             const float z = fmaf((float)(ww[q] >> 8), c2, v[4 * m + q] + c0);
             neg = __funnelshift_l(__float_as_uint(z), neg, 1);  // neg = neg << 1 | sign(z)
         }
@@ -156,34 +169,44 @@ __device__ __forceinline__ void sink_pack1(const PassParams& p, int n, uint32_t 
     dst[((i0 - lane) >> 5) + lane] = mine;
 }
 
-__device__ __forceinline__ void sink_packK(const PassParams& p, int n, uint32_t id, int64_t i0, uint32_t lane,
+// K dithers: the count c_r of non-negative signs of register r is kept bit-sliced, plane b being a
+// per-lane word whose bit r is bit b of c_r.  Each dither yields the sign mask of the 32 registers
+// (funnel shifts, as above), which a ripple of AND/XOR adds to the planes; at the end every plane
+// goes through the same warp transpose as the one-dither sink.  No per-register counters.
+__device__ __forceinline__ void sink_packK(const PassParamsRK& p, int n, uint32_t id, int64_t i0, uint32_t lane,
                                            const float (&v)[32], float amp)
 {
     const uint32_t cbase = ((uint32_t)(i0 >> 7) << 5) + lane;
     const float dc = p.dither_c * amp;
-    int cnt[32];
+    uint32_t plane[8];
 #pragma unroll
-    for (int r = 0; r < 32; ++r) cnt[r] = 0;
+    for (int b = 0; b < 8; ++b) plane[b] = 0u;
     for (int k = 0; k < p.K; ++k) {
+        uint32_t neg = 0;
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-            const uint4 w = rng_words(p.rng, id, 1u + (uint32_t)k, cbase + 32u * m);
+        for (int m = 7; m >= 0; --m) {
+            const uint4 w = rng_words_dither(p, id, 1u + (uint32_t)k, cbase + 32u * m);
             const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                cnt[4 * m + q] += (fmaf(dither_from_word(ww[q]), dc, v[4 * m + q]) >= 0.f) ? 1 : 0;
+            for (int q = 3; q >= 0; --q) {
+                const float z = fmaf(fmaf((float)(ww[q] >> 8), 2.f, -16777215.f), dc, v[4 * m + q]);
+                neg = __funnelshift_l(__float_as_uint(z), neg, 1);
+            }
+        }
+        uint32_t carry = ~neg;   // bit r: register r counts one more
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            if (b < p.P) {
+                const uint32_t t = plane[b] & carry;
+                plane[b] ^= carry;
+                carry = t;
+            }
         }
     }
     uint32_t* dst = static_cast<uint32_t*>(p.dst) + (int64_t)n * p.dst_stride + ((i0 - lane) >> 5) + lane;
-    for (int pl = 0; pl < p.P; ++pl) {
-        uint32_t mine = 0;
 #pragma unroll
-        for (int r = 0; r < 32; ++r) {
-            const uint32_t b = __ballot_sync(0xFFFFFFFFu, (cnt[r] >> pl) & 1);
-            if (lane == r) mine = b;
-        }
-        dst[(int64_t)pl * (p.dp >> 5)] = mine;
-    }
+    for (int b = 0; b < 8; ++b)
+        if (b < p.P) dst[(int64_t)b * (p.dp >> 5)] = warp_transpose_bits(plane[b], lane);
 }
 
 __device__ __forceinline__ void sink_final_store(const PassParams& p, int64_t i0, const float (&accv)[32], float amp)
@@ -209,7 +232,7 @@ __device__ __forceinline__ void sink_final_store(const PassParams& p, int64_t i0
 // row_kernel: sources read by the threads themselves (single-pass transforms)
 // =============================================================================================
 template <int T, int SRC, int SINK>
-__global__ void __launch_bounds__(1 << (T - 5), min_blocks<T, SINK>()) row_kernel(const PassParams p)
+__global__ void __launch_bounds__(1 << (T - 5), min_blocks<T, SINK>()) row_kernel(const typename KernelParams<SINK>::type p)
 {
     using C = RowCfg<T>;
     extern __shared__ __align__(16) float smem[];
@@ -316,11 +339,11 @@ __global__ void __launch_bounds__(1 << (T - 5), min_blocks<T, SINK>()) row_kerne
         load_round_L(smem, baseL, v);
         butterflies32<C::ACT_L>(v);
 
-        if (SINK == SINK_WS) {
+        if constexpr (SINK == SINK_WS) {
             sink_ws(p, n, i0, v);
-        } else if (SINK == SINK_PACK1) {
+        } else if constexpr (SINK == SINK_PACK1) {
             sink_pack1(p, n, id, i0, lane, v, s_amp);
-        } else if (SINK == SINK_PACKK) {
+        } else if constexpr (SINK == SINK_PACKK) {
             sink_packK(p, n, id, i0, lane, v, s_amp);
         } else {
             const uint32_t* const fwl = fw + ((baseL - (int)lane) >> 5);
@@ -359,7 +382,7 @@ struct StreamCfg {
 };
 
 template <int T, int SRC, int SINK>
-__global__ void __launch_bounds__(1 << (T - 5), min_blocks<T, SINK>()) row_stream_kernel(const PassParams p, const int64_t ntiles)
+__global__ void __launch_bounds__(1 << (T - 5), min_blocks<T, SINK>()) row_stream_kernel(const typename KernelParams<SINK>::type p, const int64_t ntiles)
 {
     using C = RowCfg<T>;
     using S = StreamCfg<T, SRC>;
@@ -458,11 +481,11 @@ __global__ void __launch_bounds__(1 << (T - 5), min_blocks<T, SINK>()) row_strea
         __syncthreads();   // the tile lives in registers: the work tile may be overwritten by the next round F
         butterflies32<C::ACT_L>(v);
 
-        if (SINK == SINK_WS) {
+        if constexpr (SINK == SINK_WS) {
             sink_ws(p, n, i0, v);
-        } else if (SINK == SINK_PACK1) {
+        } else if constexpr (SINK == SINK_PACK1) {
             sink_pack1(p, n, id, i0, lane, v, amp);
-        } else if (SINK == SINK_PACKK) {
+        } else if constexpr (SINK == SINK_PACKK) {
             sink_packK(p, n, id, i0, lane, v, amp);
         } else {
             const uint32_t* const fwl = fw + ((baseL - (int)lane) >> 5);
@@ -493,13 +516,13 @@ cudaError_t launch_row_one(const PassParams& p, cudaStream_t s)
             blocks = (int64_t)sms * (per_sm > 0 ? per_sm : 1);
             if (blocks > ntiles * p.nworkers) blocks = ntiles * p.nworkers;
         }
-        kern<<<(unsigned)blocks, C::NT, kSmem, s>>>(p, ntiles);
+        kern<<<(unsigned)blocks, C::NT, kSmem, s>>>(kernel_params<SINK>(p), ntiles);
     } else {
         auto kern = row_kernel<T, SRC, SINK>;
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         const dim3 grid((unsigned)ntiles, SINK == SINK_FINAL ? 1u : (unsigned)p.nworkers);
-        kern<<<grid, C::NT, C::SMEM_BYTES, s>>>(p);
+        kern<<<grid, C::NT, C::SMEM_BYTES, s>>>(kernel_params<SINK>(p));
     }
     return cudaGetLastError();
 }

@@ -108,6 +108,34 @@ def test_two_strided_passes_2p26(F, dtype):
     assert_l2_close(out.cpu().numpy(), oracle.decode_full(to_np_words(bits)[0], d, seed, step, 0, lam)[:d])
 
 
+@pytest.mark.parametrize("dtype,d,ws_workers", [(torch.float32, (1 << 24) - 12345, 3), (torch.bfloat16, (1 << 23) + 5, 2),
+                                                 (torch.float32, 1 << 24, 2)])
+def test_encoder_2p24_batches_and_ragged_tails(F, dtype, d, ws_workers):
+    # transforms of length 2^24 on several workers take the encoder whose two passes share one kernel:
+    # a ragged last row of the strided view, rows that are padding only, both input types, and a scratch
+    # buffer that holds fewer workers than the call (batches), every bit against the oracle
+    M, seed, step, id0 = 3, 909, 12, 40
+    stride = (d + 7) // 8 * 8
+    g = torch.zeros(M, stride, dtype=dtype, device=DEV)
+    g[:, :d] = torch.randn(M, d, generator=torch.Generator(device=DEV).manual_seed(d % 1000), device=DEV).to(dtype)
+    dp = F.padded_dim(d)
+    assert dp == 1 << 24
+    ws = torch.empty(F.workspace_bytes(F.OP_ENCODE, d) * ws_workers, dtype=torch.uint8, device=DEV)
+    gh = g[:, :d].cpu().double().numpy()
+    lam = oracle.lam(float(np.linalg.norm(gh, axis=1).max()), 2.0, dp)
+    bits = torch.zeros(M, dp // 32, dtype=torch.int32, device=DEV)
+    F.encode(g, d, bits, lam, seed, step, worker_id0=id0, ws=ws, worker_stride=stride)
+    torch.cuda.synchronize()
+    gb = to_np_words(bits)
+
+    def check(n):
+        ref, margin = oracle.encode(gh[n], seed, step, id0 + n, lam, want_margin=True)
+        return assert_bits_match(gb[n][None], ref, margin, lam)
+
+    pmap(check, range(M))
+    assert F.async_timeouts() == 0
+
+
 # ---- config 4 (d = 1.3e9, bf16, 64 workers): sampled coordinates at full size --------------------
 CFG4_WORKERS = (0, 1, 31, 63)
 GRID_SPLIT = 12          # global mode: samples k = k_hi * 2^12 + k_lo
@@ -273,4 +301,40 @@ def test_config4_bf16_1p3B_sampled(F, block_log2):
 
 def test_no_bounded_wait_gave_up(F):
     # the streaming kernels poll their tile copies a bounded number of times; none may have run out
+    assert F.async_timeouts() == 0
+
+
+@pytest.mark.parametrize("cfg,block_log2", [(1, 0), (2, 0), (3, 0), (3, 20)])
+def test_tensor_core_pass_matches_plain_alu_pass(F, cfg, block_log2):
+    """The strided decode pass from packed bits on the tensor cores (H_8 on packed bytes + 8-bit integer
+    products for H_128) against the oracle through the whole server side, and bit for bit against the
+    plain-ALU kernel's accumulator."""
+    from paper_2405_11095_b200 import synthetic
+    w = synthetic.WORKLOADS[cfg]
+    M = min(w.M, 4)
+    d, seed, step = w.d, 31, 7
+    dp = F.padded_dim(d, block_log2)
+    n_eff = F.transform_len(d, block_log2)
+    rng = np.random.default_rng(cfg)
+    words = rng.integers(0, 2 ** 32, (M, dp // 32), dtype=np.uint64).astype(np.uint32)
+    words[0, : dp // 64] = 0xFFFFFFFF            # long runs of equal signs: the extreme values of the small factors
+    words[1, dp // 64:] = 0
+    bits = torch.from_numpy(words.view(np.int32)).to(DEV)
+    lam = 0.37
+    ws = torch.empty(F.workspace_bytes(F.OP_AGGREGATE, d, block_log2=block_log2) * M, dtype=torch.uint8, device=DEV)
+    acc = {}
+    for on in (False, True):
+        prev = F.set_tensor_core_pass(on)
+        try:
+            a = torch.empty(dp, dtype=torch.float32, device=DEV)
+            F.server_aggregate(bits, d, a, lam, seed, step, block_log2=block_log2, ws=ws)
+            torch.cuda.synchronize()
+            acc[on] = a
+        finally:
+            F.set_tensor_core_pass(prev)
+    assert torch.equal(acc[True], acc[False])
+    gbar = np.zeros(dp)
+    for part in pmap(lambda n: oracle.decode_full(words[n], d, seed, step, n, lam, block_log2=block_log2), range(M)):
+        gbar += part
+    assert_l2_close(acc[True].cpu().numpy(), gbar / M)
     assert F.async_timeouts() == 0
