@@ -51,6 +51,10 @@ def parse_args():
                     help="run the uplink encoder's workers as this many sub-batches on side streams")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="repeat the block of --steps timed steps until this much device time has been timed")
+    ap.add_argument("--fused-encoder", action="store_true",
+                    help="run the uplink encoder of a 2^24-long transform as one kernel instead of two")
+    ap.add_argument("--tensor-core-pass", type=int, default=None, choices=[0, 1, 2, 3],
+                    help="decoder passes on the tensor cores: 1 = strided, 2 = contiguous, 3 = both (default: the library's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-legs", action="store_true", help="skip the extra workloads, the K > 1 downlink table and the issue-rate probe")
@@ -252,6 +256,8 @@ def implementation_bytes(label, dp, P):
     src, sink, workers = label_parts(label)
     per = {"f32": 4.0, "bf16": 2.0, "bits": P / 8.0, "ws": 4.0, "ws16": 2.0}[src]
     per += {"ws": 4.0, "ws16": 2.0, "pack1": 1 / 8.0, "packK": P / 8.0, "final": 0.0, "amp": 0.0}[sink]
+    if label.startswith("fused"):
+        per += 8.0   # both passes in one kernel: the fp32 intermediate is written and read inside it
     return per * workers * dp + (4.0 * dp if sink == "final" else 0.0)
 
 
@@ -267,7 +273,8 @@ def algorithmic_bytes(label, d, dp, P):
 
 
 def is_uplink_kernel(k):
-    return "f32->" in k or "bf16->" in k or "->pack" in k
+    # ("col..:ws->ws" is an encoder's middle pass, "dcol..:ws->ws" a decoder's)
+    return "f32->" in k or "bf16->" in k or "->pack" in k or (k.startswith("col") and "ws->ws" in k)
 
 
 # --------------------------------------------------------------------------- one workload on the GPU
@@ -303,7 +310,8 @@ def run_workload(env, args, w, steps, warmup, min_seconds, want_e2e):
 
     ws_per = F.workspace_bytes(F.OP_AGGREGATE, d, block_log2=b, K=w.K)
     ws_workers = args.ws_workers or R
-    ws = torch.empty(max(16, ws_per * ws_workers), dtype=torch.uint8, device=dev) if ws_per else None
+    # (+ the progress words with which the one-kernel encoder takes all its workers in one launch)
+    ws = torch.empty(max(16, ws_per * ws_workers + F.fused_sync_bytes(ws_workers)), dtype=torch.uint8, device=dev) if ws_per else None
     buf = D.RoundTripBuffers(bits=torch.zeros(R, dp // 32, dtype=torch.int32, device=dev),
                              acc=torch.zeros(dp, dtype=torch.float32, device=dev),
                              down=torch.zeros(P, dp // 32, dtype=torch.int32, device=dev),
@@ -574,6 +582,10 @@ def main():
     from paper_2405_11095_b200 import synthetic
 
     F.lib()  # fail now if the CUDA library is missing
+    if args.fused_encoder:
+        F.set_fused_encoder(True)
+    if args.tensor_core_pass is not None:
+        F.set_tensor_core_pass(args.tensor_core_pass)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -36,7 +36,11 @@
  *   - `ws` is scratch, contents undefined on entry and exit.  fosgd_workspace_bytes gives
  *     the minimum (one worker in flight); the calls that take several workers batch as many
  *     per launch as a larger `ws` allows.  Transforms that fit one thread block's tile
- *     (length <= 2^15) need none (ws may be NULL, ws_bytes 0).
+ *     (length <= 2^15) need none (ws may be NULL, ws_bytes 0).  The one-kernel encoder (see
+ *     fosgd_set_fused_encoder) keeps 16 + 4 bytes per worker of progress words behind the
+ *     intermediates: with FOSGD_FUSED_SYNC_BYTES(M) more than M times the minimum all M
+ *     workers go in one launch, with exactly M times the minimum the last worker gets a
+ *     launch of its own.
  *   - Return value: FOSGD_OK or a negative status.  On an argument, alignment, workspace,
  *     size or limit error (every status but FOSGD_ECUDA) nothing has been enqueued.
  *     FOSGD_ECUDA means a launch or a runtime call failed, possibly after earlier kernels of
@@ -229,15 +233,31 @@ int fosgd_trace_count(void);            /* launches recorded since the array was
 const char* fosgd_trace_label(int k);   /* e.g. "col10:f32->ws@4", "row14:ws->pack1@4", "row14:ws16->final@srv" (kernel, source->sink,
                                            workers of the launch, or "srv" for the server's own vector on the downlink); valid until the next call */
 
-/* Kernel choice for the ten strided stages of a decoder that starts from one packed plane (transform
- * lengths 2^20 .. 2^25: fosgd_decode, fosgd_server_aggregate, and the downlink decoder with K = 1).
- * The recursion H_k = H_1 (x) H_{k-1} below Def. 3.4 makes H_1024 = H_8 (x) H_128 a legal factor; with
- * on != 0 those stages run as H_8 on packed bytes plus a 128 x 128 x 128 8-bit integer product per
- * block on the tensor cores (tcgen05, accumulators in tensor memory), otherwise in packed fp16
- * arithmetic on the plain ALUs.  Both give the same fp16 intermediate bit for bit (the values are
- * integers of magnitude <= 1024).  Default 0: measured on a B200, the plain-ALU kernel is the faster
- * of the two.  Process-wide; returns the previous setting. */
-int fosgd_set_tensor_core_pass(int on);
+/* Which passes of a decoder that starts from one packed plane (fosgd_decode, fosgd_server_aggregate,
+ * the downlink decoder with K = 1; transform lengths 2^20 .. 2^25) run on the tensor cores.  The
+ * recursion H_k = H_1 (x) H_{k-1} below Def. 3.4 makes every Kronecker factor H_128 a legal 128 x 128
+ * matrix product, and on the decode side all operands are exact small integers (Def. 3.8: q_i = +-1).
+ *   FOSGD_TC_STRIDED     the ten strided stages as H_8 on packed bytes plus a 128 x 128 x 128 8-bit integer
+ *                        product per block (tcgen05 kind::i8), instead of packed fp16 arithmetic on the
+ *                        plain ALUs;
+ *   FOSGD_TC_CONTIGUOUS  the contiguous pass on tiles of 2^14 (transform length 2^24) as H_4 in packed
+ *                        fp16 while staging, a 128 x 128 x 128 fp16 product with fp32 accumulators in tensor
+ *                        memory per tile and worker (tcgen05 kind::f16), and H_32, flip and the sum over
+ *                        the workers in registers, instead of fp32 butterflies on the plain ALUs.
+ * Either way the results are the same bit for bit (all values are integers below 2^24 in magnitude).
+ * Default: FOSGD_TC_CONTIGUOUS (the choices measured faster on a B200).  Process-wide; returns the
+ * previous mask. */
+enum { FOSGD_TC_STRIDED = 1, FOSGD_TC_CONTIGUOUS = 2 };
+int fosgd_set_tensor_core_pass(int mask);
+
+/* Kernel choice for the uplink encoder of fp32 gradients when the transform length is 2^24 (ten strided
+ * stages, then contiguous tiles of 2^14).  With on != 0 (the default) both passes run as one persistent
+ * kernel: half of every thread block stages strided tiles through the tensor copy engine while the other
+ * half transforms, dithers and packs the contiguous tiles of workers whose strided pass is complete, so
+ * that the memory-bound and the issue-bound half of the encoder overlap.  With on == 0 the two passes run
+ * as two kernels, one after the other.  Same bits either way.  Process-wide; returns the previous setting. */
+int fosgd_set_fused_encoder(int on);
+#define FOSGD_FUSED_SYNC_BYTES(M) ((((size_t)(M) + 4) * 4 + 15) & ~(size_t)15)
 
 /* Issue-rate probe (measurement aid; no counterpart in the paper).  Enqueues one kernel that
  * keeps every scheduler of every SM busy with independent register-resident chains of one

@@ -26,7 +26,8 @@ EXPORTS = ("fosgd_padded_dim", "fosgd_planes", "fosgd_lambda", "fosgd_lambda_ser
            "fosgd_last_cuda_error", "fosgd_version", "fosgd_trace_passes", "fosgd_trace_count",
            "fosgd_trace_label", "fosgd_decode_noalloc", "fosgd_async_timeouts", "fosgd_amplitudes",
            "fosgd_encode_dev", "fosgd_server_aggregate_dev", "fosgd_downlink_decode_dev", "fosgd_downlink_apply",
-           "fosgd_downlink_encode", "fosgd_probe_issue_rate", "fosgd_set_tensor_core_pass")
+           "fosgd_downlink_encode", "fosgd_probe_issue_rate", "fosgd_set_tensor_core_pass",
+           "fosgd_set_fused_encoder")
 
 
 class FosgdError(RuntimeError):
@@ -68,6 +69,7 @@ def _load() -> C.CDLL:
     L.fosgd_downlink_decode_dev.argtypes = [vp, i64, u64, u64, vp, cint, cint, cint, vp, vp, sz, vp]
     L.fosgd_probe_issue_rate.argtypes = [cint, cint, C.POINTER(dbl), vp, vp]
     L.fosgd_set_tensor_core_pass.argtypes, L.fosgd_set_tensor_core_pass.restype = [cint], cint
+    L.fosgd_set_fused_encoder.argtypes, L.fosgd_set_fused_encoder.restype = [cint], cint
     L.fosgd_strerror.argtypes, L.fosgd_strerror.restype = [cint], C.c_char_p
     L.fosgd_last_cuda_error.restype = cint
     L.fosgd_version.restype = C.c_char_p
@@ -265,10 +267,26 @@ def downlink_apply(down_bits, d, x, lam_s, seed, step, step_size, K=1, block_log
     return x
 
 
-def set_tensor_core_pass(on: bool) -> bool:
-    """fosgd_set_tensor_core_pass: run the strided decode pass from packed bits on the tensor cores
-    (True) or on the plain ALUs (False, the default and the faster one); returns the previous setting."""
-    return bool(_lib.fosgd_set_tensor_core_pass(int(bool(on))))
+TC_STRIDED, TC_CONTIGUOUS = 1, 2
+
+
+def set_tensor_core_pass(mask: int) -> int:
+    """fosgd_set_tensor_core_pass: which decoder passes from one packed plane run on the tensor cores
+    (TC_STRIDED | TC_CONTIGUOUS bits; True = the strided pass only, as in its first form); returns the
+    previous mask."""
+    return int(_lib.fosgd_set_tensor_core_pass(int(mask)))
+
+
+def set_fused_encoder(on: bool) -> bool:
+    """fosgd_set_fused_encoder: run the uplink encoder of a 2^24-long transform as one kernel (True, the
+    default) or as its two passes one after the other (False); returns the previous setting."""
+    return bool(_lib.fosgd_set_fused_encoder(int(bool(on))))
+
+
+def fused_sync_bytes(M: int) -> int:
+    """FOSGD_FUSED_SYNC_BYTES: scratch beyond M * workspace_bytes(OP_ENCODE, ...) with which the one-kernel
+    encoder takes all M workers in one launch."""
+    return ((M + 4) * 4 + 15) & ~15
 
 
 PROBE_FADD, PROBE_FFMA, PROBE_LOP3, PROBE_IMAD = range(4)

@@ -26,7 +26,8 @@ def _nvcc() -> str:
 def _units():
     units = [("api.cu", "api.o", []), ("col_kernels.cu", "col_kernels.o", []),
              ("small_kernels.cu", "small_kernels.o", []), ("noalloc.cu", "noalloc.o", []), ("amplitudes.cu", "amplitudes.o", []),
-             ("probe.cu", "probe.o", []), ("tc_kernels.cu", "tc_kernels.o", [])]
+             ("probe.cu", "probe.o", []), ("tc_kernels.cu", "tc_kernels.o", []),
+             ("fused_encode.cu", "fused_encode.o", []), ("tc_row_kernels.cu", "tc_row_kernels.o", [])]
     units += [("row_inst.cu", f"row_{t}.o", [f"-DFOSGD_ROW_T={t}"]) for t in ROW_TILES]
     return units
 

@@ -43,27 +43,40 @@ thread_local int g_last_cuda_error = 0;
 
 // Optional per-launch timing hooks (fosgd_trace_passes): caller-owned events, recorded around
 // every kernel launch issued by this thread.
-struct TraceEntry { char kind; int size, src, sink, workers; };   // workers = 0: the server's own vector (downlink)
+struct TraceEntry { char kind; int size, src, sink, workers; bool decoder; };   // workers = 0: the server's own vector (downlink)
 thread_local cudaEvent_t* g_trace_events = nullptr;
 thread_local int g_trace_capacity = 0;
 thread_local int g_trace_count = 0;
 thread_local TraceEntry g_trace_log[64];
 thread_local char g_trace_label[48];
 
-cudaError_t traced(char kind, int size, int src, int sink, const PassParams& p, cudaStream_t s)
+bool trace_begin(cudaStream_t s)
 {
     const bool on = g_trace_events != nullptr && g_trace_count < g_trace_capacity && g_trace_count < 64;
     if (on) cudaEventRecord(g_trace_events[2 * g_trace_count], s);
+    return on;
+}
+
+void trace_end(bool on, cudaStream_t s, const TraceEntry& entry)
+{
+    if (!on) return;
+    cudaEventRecord(g_trace_events[2 * g_trace_count + 1], s);
+    g_trace_log[g_trace_count] = entry;
+    ++g_trace_count;
+}
+
+// decoder: the pass belongs to a transform that ends in the flip + sum sink (tells the intermediate passes
+// of the two directions apart in the trace)
+cudaError_t traced(char kind, int size, int src, int sink, const PassParams& p, cudaStream_t s, bool decoder = false)
+{
+    const bool on = trace_begin(s);
     cudaError_t e = kind == 'r' ? launch_row(size, src, sink, p, s)
                   : kind == 'c' ? launch_col(size, src, p, s)
                   : kind == 'h' ? launch_colh(size, p, s)
                   : kind == 't' ? launch_tc_col(p, s)
+                  : kind == 'u' ? launch_tc_row(p, s)
                                 : launch_small(size, src, sink, p, s);
-    if (on) {
-        cudaEventRecord(g_trace_events[2 * g_trace_count + 1], s);
-        g_trace_log[g_trace_count] = TraceEntry{kind, size, src, sink, p.id0 == FOSGD_SERVER_ID ? 0 : p.nworkers};
-        ++g_trace_count;
-    }
+    trace_end(on, s, TraceEntry{kind, size, src, sink, p.id0 == FOSGD_SERVER_ID ? 0 : p.nworkers, decoder});
     return e;
 }
 
@@ -168,8 +181,13 @@ Rng make_rng(uint64_t seed, uint64_t step)
 
 // which kernel runs the ten strided stages of a decoder whose source is one packed plane: 0 = packed
 // fp16 arithmetic on the plain ALUs (the faster one as measured, hence the default), 1 = tensor cores
-std::atomic<int> g_tensor_core_pass{0};
-bool tc_enabled() { return g_tensor_core_pass.load(std::memory_order_relaxed) != 0; }
+std::atomic<int> g_tensor_core_pass{FOSGD_TC_CONTIGUOUS};
+bool tc_enabled() { return (g_tensor_core_pass.load(std::memory_order_relaxed) & FOSGD_TC_STRIDED) != 0; }
+bool tc_row_enabled() { return (g_tensor_core_pass.load(std::memory_order_relaxed) & FOSGD_TC_CONTIGUOUS) != 0; }
+// whether an encoder of ten strided stages + a 2^14 tile runs as the one-kernel form or as two kernels (default:
+// measured on a B200 the two kernels are the faster form)
+std::atomic<int> g_fused_encoder{0};
+bool fused_encoder_enabled() { return g_fused_encoder.load(std::memory_order_relaxed) != 0; }
 
 // Enqueue one source -> sink transform for p.nworkers workers.  Workers are processed in
 // chunks of as many as the scratch buffer holds; SINK_FINAL accumulates chunk after chunk.
@@ -186,7 +204,17 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
     if (ws == nullptr || ws_bytes < g.ws_per_worker) return FOSGD_EWORKSPACE;
     const size_t cap = ws_bytes / g.ws_per_worker;
     const int total = p.nworkers;
-    const int chunk = (int)(cap < (size_t)total ? cap : (size_t)total);
+    int chunk = (int)(cap < (size_t)total ? cap : (size_t)total);
+    // The one-kernel encoder (fused_encode.cu) keeps its ticket and progress words behind the chunk's
+    // intermediates.  Scratch sized for exactly `chunk` workers has no room for them: the chunk then gives up
+    // its last worker's slot (a caller who adds enc_fused_sync_bytes to the scratch keeps the full chunk).
+    const bool fused_geometry = src == SRC_G32 && sink == SINK_PACK1 && pl.ncol == 1 && pl.A[0] == 10 && pl.T == 14 &&
+                                fused_encoder_enabled();
+    bool fused = false;
+    if (fused_geometry) {
+        if (ws_bytes - (size_t)chunk * g.ws_per_worker >= enc_fused_sync_bytes(chunk)) fused = true;
+        else if (chunk >= 2) { --chunk; fused = true; }
+    }
     const float final_scale = p.scale;
     const int first_overwrite = p.overwrite;
     const char* src0 = static_cast<const char*>(p.src);
@@ -202,6 +230,24 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
         if (p.amp_dev) q.amp_dev = p.amp_dev + (int64_t)n0 * p.amp_stride;
         const void* const srck = src0 + (size_t)n0 * (size_t)p.src_stride * src_elem_bytes(src);
         bool tensor_pass = false;
+        if (fused) {
+            PassParams pc = q, pr = q;
+            pc.src = srck;
+            pc.dst = ws;
+            pc.dst_stride = g.dp;
+            pc.lo_log = pl.lo[0];
+            pr.src = ws;
+            pr.src_stride = g.dp;
+            pr.dst = dst0 + (size_t)n0 * (size_t)p.dst_stride * sink_elem_bytes(sink);
+            bool launched = false;
+            const bool on = trace_begin(s);
+            e = launch_enc_fused(pc, pr, pl.T, pl.A[0], reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + (size_t)chunk * g.ws_per_worker),
+                                 s, &launched);
+            if (launched) trace_end(on, s, TraceEntry{'f', pl.L, src, sink, p.id0 == FOSGD_SERVER_ID ? 0 : m, false});
+            if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
+            if (launched) continue;
+            // (not launched: nothing was recorded or enqueued besides the start event, which the next pass re-records)
+        }
         if (half_path) {
             PassParams pc = q;
             pc.src = srck;
@@ -222,7 +268,7 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
                 pc.dst = ws;
                 pc.dst_stride = g.dp;
                 pc.lo_log = pl.lo[c];
-                FOSGD_CUDA_OK(traced('c', pl.A[c], first ? src : (int)SRC_WS, SINK_WS, pc, s));
+                FOSGD_CUDA_OK(traced('c', pl.A[c], first ? src : (int)SRC_WS, SINK_WS, pc, s, sink == SINK_FINAL));
             }
         }
         PassParams pr = q;
@@ -235,7 +281,10 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
         } else {
             pr.dst = dst0 + (size_t)n0 * (size_t)p.dst_stride * sink_elem_bytes(sink);
         }
-        FOSGD_CUDA_OK(traced('r', pl.T, half_path ? (int)SRC_WS16 : (int)SRC_WS, sink, pr, s));
+        if (half_path && sink == SINK_FINAL && tc_row_enabled() && tc_row_applicable(pr, pl.T))
+            FOSGD_CUDA_OK(traced('u', pl.T, SRC_WS16, sink, pr, s));
+        else
+            FOSGD_CUDA_OK(traced('r', pl.T, half_path ? (int)SRC_WS16 : (int)SRC_WS, sink, pr, s));
     }
 #undef FOSGD_CUDA_OK
     return FOSGD_OK;
@@ -573,7 +622,7 @@ int fosgd_amplitudes(const void* grads, int dtype, int64_t d, int64_t worker_str
                                       (cudaStream_t)stream);
     if (on) {
         cudaEventRecord(g_trace_events[2 * g_trace_count + 1], (cudaStream_t)stream);
-        g_trace_log[g_trace_count] = TraceEntry{'n', g.L, dtype == FOSGD_BF16 ? 1 : 0, 5, M};
+        g_trace_log[g_trace_count] = TraceEntry{'n', g.L, dtype == FOSGD_BF16 ? 1 : 0, 5, M, false};
         ++g_trace_count;
     }
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
@@ -604,10 +653,14 @@ int fosgd_async_timeouts(int* count)
     int total = 0;
     {
         int t = 0;
+        int f = 0;
         cudaError_t e = col_timeouts(&total);
         if (e == cudaSuccess) e = tc_timeouts(&t);
+        int u = 0;
+        if (e == cudaSuccess) e = fused_timeouts(&f);
+        if (e == cudaSuccess) e = tcrow_timeouts(&u);
         if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
-        total += t;
+        total += t + f + u;
     }
     for (auto fn : fns) {
         int c = 0;
@@ -640,14 +693,19 @@ const char* fosgd_trace_label(int k)
     if (t.workers > 0) snprintf(who, sizeof who, "%d", t.workers);
     else snprintf(who, sizeof who, "srv");
     snprintf(g_trace_label, sizeof g_trace_label, "%s%d:%s->%s@%s",
-             t.kind == 'r' ? "row" : (t.kind == 'c' ? "col" : (t.kind == 'h' ? "colh" : (t.kind == 'n' ? "norm" : (t.kind == 't' ? "tc" : "small")))), t.size, srcs[t.src], sinks[t.sink],
-             who);
+             t.kind == 'r' ? "row" : (t.kind == 'c' ? (t.decoder ? "dcol" : "col") : (t.kind == 'h' ? "colh" : (t.kind == 'n' ? "norm" : (t.kind == 't' ? "tc" : (t.kind == 'u' ? "tcrow" : (t.kind == 'f' ? "fused" : "small")))))),
+             t.size, srcs[t.src], sinks[t.sink], who);
     return g_trace_label;
 }
 
-int fosgd_set_tensor_core_pass(int on)
+int fosgd_set_tensor_core_pass(int mask)
 {
-    return g_tensor_core_pass.exchange(on ? 1 : 0, std::memory_order_relaxed);
+    return g_tensor_core_pass.exchange(mask & (FOSGD_TC_STRIDED | FOSGD_TC_CONTIGUOUS), std::memory_order_relaxed);
+}
+
+int fosgd_set_fused_encoder(int on)
+{
+    return g_fused_encoder.exchange(on ? 1 : 0, std::memory_order_relaxed);
 }
 
 const char* fosgd_version(void) { return "libfosgd 0.1 (sm_100a)"; }

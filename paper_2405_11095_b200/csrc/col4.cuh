@@ -32,6 +32,23 @@ __device__ __forceinline__ float flip_at(float x, uint32_t word, uint32_t sh)
     return __uint_as_float(__float_as_uint(x) ^ ((word << sh) & 0x80000000u));
 }
 
+// How the 512 threads of a run meet: the whole block (the stand-alone kernel), or one group of a larger
+// block on a named barrier (the fused encoder, where another group works beside this one).
+struct BlockSync {
+    static __device__ __forceinline__ void sync() { __syncthreads(); }
+    static __device__ __forceinline__ bool all(bool ok) { return __syncthreads_and(ok ? 1 : 0) != 0; }
+};
+template <int ID, int NTHREADS>
+struct GroupSync {
+    static __device__ __forceinline__ void sync() { group_sync(ID, NTHREADS); }
+    static __device__ __forceinline__ bool all(bool ok) { return group_all(ID, NTHREADS, ok); }
+};
+
+// Tensor map over fp32 gradients as a strided pass of ten stages sees them: (S columns, whole rows, workers),
+// boxes of 16 columns x 256 rows.  False if the driver entry point is missing or refuses the geometry.
+bool make_col_tensor_map(CUtensorMap* map, const void* base, uint64_t S, uint64_t rows, uint64_t workers,
+                         uint64_t worker_stride_elems);
+
 struct Col4 {
     static constexpr int A = 10, ROWS = 1 << A, RUN = 8, THREADS = 512;
     static constexpr int NBUF = 2;   // landing buffers (copies in flight ahead of the tile being transformed)
@@ -41,8 +58,10 @@ struct Col4 {
 };
 
 // One run: tiles seg0 .. seg0 + 7 (16-column segments of the matrix view) of worker n, by the 512 threads
-// of a block.  timeouts: device counter bumped when a bounded wait gave up.
-__device__ __forceinline__ void col4_run(const PassParams& p, const CUtensorMap* tmap, const uint32_t full_rows, const int n,
+// of a block or group (tid = 0 .. 511).  timeouts: device counter bumped when a bounded wait gave up;
+// the return value says whether the run completed (the same for all threads).
+template <typename S>
+__device__ __forceinline__ bool col4_run(const PassParams& p, const CUtensorMap* tmap, const uint32_t full_rows, const int n,
                                          const uint32_t seg0, unsigned char* smem_raw, const int tid, int* timeouts)
 {
     using C = Col4;
@@ -63,9 +82,10 @@ __device__ __forceinline__ void col4_run(const PassParams& p, const CUtensorMap*
 #pragma unroll
         for (int b = 0; b < NBUF; ++b) mbar_init(full + b, 1);
     }
-    __syncthreads();
+    S::sync();
 
     int issued = 0, taken = 0;   // thread 0 only
+    bool completed = true;
     auto issue = [&](int t) {
         uint64_t* const bar_full = full + (t % NBUF);
         const uint32_t dst0 = smem_u32(land0 + (t % NBUF) * LAND_BYTES);
@@ -91,13 +111,14 @@ __device__ __forceinline__ void col4_run(const PassParams& p, const CUtensorMap*
             reinterpret_cast<uint4*>(flips)[row] = rng_words(p.rng, id, 0u, (i_run + row * step) >> 7);
         }
     }
-    __syncthreads();
+    S::sync();
 
     for (int t = 0; t < RUN; ++t) {
         float* const buf = reinterpret_cast<float*>(land0 + (t % NBUF) * LAND_BYTES);
         // bounded wait; the block then agrees on the outcome, so that it stops as a whole
-        if (!__syncthreads_and(mbar_wait(full + (t % NBUF), (uint32_t)((t / NBUF) & 1)) ? 1 : 0)) {
+        if (!S::all(mbar_wait(full + (t % NBUF), (uint32_t)((t / NBUF) & 1)))) {
             if (tid == 0) atomicAdd(timeouts, 1);
+            completed = false;
             break;
         }
         if (tid == 0) ++taken;
@@ -109,7 +130,7 @@ __device__ __forceinline__ void col4_run(const PassParams& p, const CUtensorMap*
                     const uint32_t i = full_rows * step + lo_run + 16u * t + (uint32_t)tid;
                     if (i < d32) buf[(row_p << 4) + tid] = (static_cast<const float*>(p.src) + (int64_t)n * p.src_stride)[i];
                 }
-                __syncthreads();
+                S::sync();
             }
         }
         float v[32];
@@ -132,7 +153,7 @@ __device__ __forceinline__ void col4_run(const PassParams& p, const CUtensorMap*
                     make_float4(v[4 * g + 0], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
             }
         }
-        __syncthreads();
+        S::sync();
         // ---- round 2: row bits 4..6 ----
         {
             float* const p2 = buf + ((((u >> 3) << 7) | ((u & 7u) << 1) | r0) << 4) + 4u * kq;
@@ -146,7 +167,7 @@ __device__ __forceinline__ void col4_run(const PassParams& p, const CUtensorMap*
             for (int g = 0; g < 8; ++g)
                 *reinterpret_cast<float4*>(p2 + (g << 8)) = make_float4(v[4 * g + 0], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
         }
-        __syncthreads();
+        S::sync();
         // ---- round 3: row bits 1..3, then row bit 0 across lanes ----
         {
             const float* const p3 = buf + (((u << 4) | r0) << 4) + 4u * kq;
@@ -157,7 +178,7 @@ __device__ __forceinline__ void col4_run(const PassParams& p, const CUtensorMap*
             }
         }
         fence_generic_before_async();   // this thread's stores into the buffer, before the copy engine reuses it
-        __syncthreads();                // the tile lives in registers
+        S::sync();                // the tile lives in registers
         if (tid == 0 && t + NBUF < RUN) issue(t + NBUF);
         butterflies32<28>(v);
         const float sgn = r0 ? -1.f : 1.f;
@@ -172,12 +193,13 @@ __device__ __forceinline__ void col4_run(const PassParams& p, const CUtensorMap*
     // In a healthy run every issued copy has been taken; after a timeout the copies still in flight get
     // one more bounded wait, so that the engine is not left writing into shared memory that the next
     // block of this SM may own.
-    __syncthreads();
+    S::sync();
     if (tid == 0) {
         for (int k = taken; k < issued; ++k) mbar_wait(full + (k % NBUF), (uint32_t)((k / NBUF) & 1));
 #pragma unroll
         for (int b = 0; b < NBUF; ++b) mbar_inval(full + b);
     }
+    return completed;
 }
 
 // ---- the same transform by two groups of 512 threads that take tiles in turn --------------------

@@ -242,8 +242,8 @@ __global__ void __launch_bounds__(512, 2) col4_kernel(const PassParams p, const 
                                                       const int nruns, const uint32_t full_rows)
 {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    col4_run(p, &tmap, full_rows, (int)(blockIdx.x / (unsigned)nruns), (blockIdx.x % (unsigned)nruns) * 8u, smem_raw,
-             (int)threadIdx.x, &g_col_wait_timeouts);
+    col4_run<BlockSync>(p, &tmap, full_rows, (int)(blockIdx.x / (unsigned)nruns), (blockIdx.x % (unsigned)nruns) * 8u, smem_raw,
+                        (int)threadIdx.x, &g_col_wait_timeouts);
 }
 
 __global__ void __launch_bounds__(1024, 1) col4_duo_kernel(const PassParams p, const __grid_constant__ CUtensorMap tmap,
@@ -257,8 +257,8 @@ cudaError_t col_timeouts(int* out) { return cudaMemcpyFromSymbol(out, g_col_wait
 
 // Tensor map over the gradients as the strided pass sees them: (S columns, whole rows, workers).
 // False if the driver entry point is missing or refuses the geometry; the caller then uses the plain kernel.
-static bool make_col_tensor_map(CUtensorMap* map, const void* base, uint64_t S, uint64_t rows, uint64_t workers,
-                                uint64_t worker_stride_elems)
+bool make_col_tensor_map(CUtensorMap* map, const void* base, uint64_t S, uint64_t rows, uint64_t workers,
+                         uint64_t worker_stride_elems)
 {
     using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

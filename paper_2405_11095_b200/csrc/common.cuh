@@ -259,6 +259,14 @@ cudaError_t launch_colh(int A, const PassParams& p, cudaStream_t s);   // one-pl
 bool tc_col_applicable(const PassParams& p);                            // ten strided stages from one plane on the tensor cores
 cudaError_t launch_tc_col(const PassParams& p, cudaStream_t s);          // one-plane bits -> fp16 intermediate
 cudaError_t tc_timeouts(int* out);
+bool tc_row_applicable(const PassParams& p, int T);                     // contiguous 2^14 tiles of the fp16 intermediate, seven stages on the tensor cores
+cudaError_t launch_tc_row(const PassParams& p, cudaStream_t s);          // fp16 intermediate -> flip + sum sink
+cudaError_t tcrow_timeouts(int* out);
+// uplink encoder of a 2^24-long transform as one kernel (strided and contiguous pass side by side)
+size_t enc_fused_sync_bytes(int nworkers);                               // zeroed device words the launch needs
+cudaError_t launch_enc_fused(const PassParams& pc, const PassParams& pr, int T, int A, uint32_t* sync, cudaStream_t s,
+                             bool* launched);
+cudaError_t fused_timeouts(int* out);
 cudaError_t col_timeouts(int* out);                                      // synchronising read of the strided unit's counter
 cudaError_t launch_small(int L, int src, int sink, const PassParams& p, cudaStream_t s);
 cudaError_t launch_amplitudes(const void* grads, int bf16, int64_t d, int64_t worker_stride, int M, double alpha,

@@ -1,0 +1,358 @@
+// Contiguous pass of a decoder (14 stages on tiles of 2^14 coordinates, flip, sum over the workers)
+// with seven of the stages on the tensor cores (tcgen05, sm_100a).
+//
+// The source is the fp16 intermediate of the strided pass: integers of magnitude <= 1024.  A tile
+// of 2^14 consecutive coordinates is read as a matrix X of 128 rows (index bits 7..13) x 128 columns
+// (bits 0..6).  By the recursion H_k = H_1 (x) H_{k-1}, H_{2^14} = H_128 (x) H_4 (x) H_32:
+//   1. H_4 over column bits 5, 6 runs in packed fp16 on the plain ALUs while the tile is staged
+//      (values <= 4096: still exact in fp16);
+//   2. H_128 over the row bits is one 128 x 128 x 128 product D = H_128 Z per tile and worker:
+//      fp16 operands in shared memory (A = H_128, K-major; B = Z as staged, columns contiguous, i.e.
+//      MN-major), fp32 accumulators in tensor memory (exact: |D| <= 2^19), eight tcgen05.mma of K = 16
+//      issued by one thread, completion through mbarriers;
+//   3. H_32 over column bits 0..4 runs in fp32 registers: tcgen05.ld hands every thread 32
+//      consecutive columns of one row, which is also one word of the flip vector, so the flip and
+//      the sum over the workers follow in the same registers.
+// All values are integers below 2^24 in magnitude, so the result equals the plain-ALU kernel's bit
+// for bit.
+//
+// A block is 16 worker warps and one warp that issues the products.  It keeps a tile position and
+// walks the workers (sums in registers), then moves to its next tile.  Per item (tile, worker) a
+// worker warp stages its share of Z into one of two operand buffers, then drains the accumulator of
+// the previous item while the product of this one runs.  Synchronisation is by mbarriers only
+// (operand full / free, accumulator full / free, flips ready); every wait is bounded.
+#include "common.cuh"
+
+namespace fosgd {
+
+static __device__ int g_tcrow_wait_timeouts;   // warps that abandoned a bounded wait
+
+namespace {
+
+constexpr int kT = 14;
+constexpr int kWorkerWarps = 16;
+constexpr int kThreads = (kWorkerWarps + 1) * 32;
+constexpr uint32_t kAChunkStride = 128;                    // bytes between core matrices along K
+constexpr uint32_t kAGroupStride = 16 * 128;               // bytes between groups of eight rows of A
+constexpr uint32_t kBGroupStride = 16 * 128 + 32;          // bytes between groups of eight columns of B (+32: staging stores hit distinct banks)
+constexpr uint32_t kOffA = 0;                              // H_128 as fp16: 32 KiB
+constexpr uint32_t kOffB = 32768;                          // two operand buffers
+constexpr uint32_t kBBytes = 16 * kBGroupStride;
+constexpr uint32_t kOffFlips = kOffB + 2 * kBBytes;        // two buffers of 128 rows x 4 flip words
+constexpr uint32_t kOffBar = kOffFlips + 2 * 2048;         // ten mbarriers, stop word, tensor-memory base
+constexpr uint32_t kSmemBytes = kOffBar + 128;
+
+enum { BAR_B_FULL = 0, BAR_B_FREE = 2, BAR_ACC_FULL = 4, BAR_ACC_FREE = 6, BAR_FLIPS = 8 };
+
+// instruction descriptor: D = f32 (1 << 4), A = B = fp16 (0), A K-major, B MN-major (1 << 16), N = 128, M = 128
+constexpr uint32_t kIdescF16 = (1u << 4) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+// shared-memory matrix descriptor, no swizzle: start address, leading and stride byte offsets in
+// units of 16 bytes, descriptor version 1
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(sbo_bytes >> 4) << 32) | ((uint64_t)1 << 46);
+}
+
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescF16), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint64_t* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// bounded wait that also gives up when the block's stop word is raised
+__device__ __forceinline__ bool mbar_wait_or_stop(uint64_t* bar, uint32_t parity, const volatile int* stop)
+{
+    for (int it = 0; it < (1 << 22); ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (done) return true;
+        if ((it & 255) == 255 && *stop) return false;
+    }
+    return false;
+}
+
+// 32 consecutive accumulator columns of this thread's lane
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t u[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+          "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
+          "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
+          "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int r = 0; r < 32; ++r) v[r] = __uint_as_float(u[r]);
+}
+
+__device__ __forceinline__ void hbutterfly(uint4& a, uint4& b)
+{
+    __half2* const pa = reinterpret_cast<__half2*>(&a);
+    __half2* const pb = reinterpret_cast<__half2*>(&b);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const __half2 x = pa[k], y = pb[k];
+        pa[k] = __hadd2(x, y);
+        pb[k] = __hsub2(x, y);
+    }
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassParams p, const int ntiles)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const uint32_t lane = tid & 31;
+    uint64_t* const bar = reinterpret_cast<uint64_t*>(smem + kOffBar);
+    volatile int* const s_stop = reinterpret_cast<volatile int*>(smem + kOffBar + 96);
+    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 100);
+
+    // ---- once per block: the constant operand, barriers, tensor memory ----
+    if (tid < 512) {
+        // A[m][k] = (-1)^popcount(m & k) as fp16, K-major core matrices of 8 rows x 16 bytes: thread = (row m, 32 of its k)
+        const uint32_t m = (uint32_t)tid >> 2, k0 = ((uint32_t)tid & 3u) * 32u;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t w[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t k = k0 + 8u * c + 2u * q;
+                const uint32_t lo = (__popc(m & k) & 1) ? 0xBC00u : 0x3C00u;
+                const uint32_t hi = (__popc(m & (k + 1u)) & 1) ? 0xBC00u : 0x3C00u;
+                w[q] = lo | (hi << 16);
+            }
+            *reinterpret_cast<uint4*>(smem + kOffA + (m & 7u) * 16u + (m >> 3) * kAGroupStride + ((k0 >> 3) + c) * kAChunkStride) =
+                make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+    if (warp == kWorkerWarps) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar + BAR_B_FULL + b, kWorkerWarps);
+            mbar_init(bar + BAR_B_FREE + b, 1);
+            mbar_init(bar + BAR_ACC_FULL + b, 1);
+            mbar_init(bar + BAR_ACC_FREE + b, kWorkerWarps);
+            mbar_init(bar + BAR_FLIPS + b, 4);
+        }
+        *s_stop = 0;
+    }
+    fence_generic_before_async();   // the constant operand, for the tensor core's reads
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int W = p.nworkers;
+    const int my_tiles = ((int)blockIdx.x < ntiles) ? (ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    const int64_t nitems = (int64_t)my_tiles * W;   // item g: tile blockIdx.x + (g / W) * gridDim.x, worker g % W
+
+    if (warp == kWorkerWarps) {
+        // ================= the warp that issues the products =================
+        if (lane == 0) {
+            const uint64_t adesc = umma_desc(smem_u32(smem + kOffA), kAChunkStride, kAGroupStride);
+            bool ok = true;
+            int64_t g = 0;
+            for (; g < nitems; ++g) {
+                const uint32_t b = (uint32_t)g & 1u, u = (uint32_t)(g >> 1);
+                ok = mbar_wait_or_stop(bar + BAR_B_FULL + b, u & 1u, s_stop);                        // operand staged
+                if (ok && u > 0) ok = mbar_wait_or_stop(bar + BAR_ACC_FREE + b, (u - 1u) & 1u, s_stop);   // accumulator drained
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t bdesc = umma_desc(smem_u32(smem + kOffB + b * kBBytes), 128u, kBGroupStride);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)   // K = 16 per instruction: two 16-byte chunks of A, two groups of eight rows of B
+                    umma_f16(tmem_base + b * 128u, adesc + (uint64_t)(ks * (256 >> 4)), bdesc + (uint64_t)(ks * (256 >> 4)), ks > 0 ? 1u : 0u);
+                umma_commit(bar + BAR_B_FREE + b);
+                umma_commit(bar + BAR_ACC_FULL + b);
+            }
+            if (!ok) {
+                if (atomicExch((int*)s_stop, 1) == 0) atomicAdd(&g_tcrow_wait_timeouts, 1);
+                // products already committed may still be running: one more bounded wait each before the tensor memory goes back
+                for (int64_t h = (g >= 2 ? g - 2 : 0); h < g; ++h) mbar_wait(bar + BAR_ACC_FULL + (h & 1), (uint32_t)(h >> 1) & 1u);
+            }
+        }
+    } else {
+        // ================= worker warps: stage, drain, flip, sum =================
+        const uint32_t srow = (uint32_t)tid >> 2, sq = (uint32_t)tid & 3u;       // staging role: row of the tile, column chunks sq + 4 t
+        const uint32_t lq = (uint32_t)warp & 3u, cw = (uint32_t)warp >> 2;       // drain role: lane quarter, 32 of the 128 columns
+        const uint32_t jrow = lq * 32u + lane;                                  // output row (index bits 7..13)
+        float accv[32];
+        uint4 pre[4];
+        bool ok = true;
+
+        // where an item sits: first coordinate of its tile and its worker; advanced item by item (worker fastest)
+        struct Cursor {
+            int64_t tile_base;
+            int n;
+        };
+        const int64_t tile_step = (int64_t)gridDim.x << kT;
+        auto advance = [&](Cursor& c) {
+            if (++c.n == W) {
+                c.n = 0;
+                c.tile_base += tile_step;
+            }
+        };
+        Cursor c_load{(int64_t)blockIdx.x << kT, 0}, c_stage = c_load, c_drain = c_load;
+        auto load_item = [&]() {
+            const __half* const src = static_cast<const __half*>(p.src) + (int64_t)c_load.n * p.src_stride + c_load.tile_base + srow * 128u + sq * 8u;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) pre[t] = __ldcs(reinterpret_cast<const uint4*>(src + 32 * t));
+            advance(c_load);
+        };
+        // stage item g from `pre` into its operand buffer (and, warps 0..3, its flip words)
+        auto stage_item = [&](int64_t g) -> bool {
+            const uint32_t b = (uint32_t)g & 1u, u = (uint32_t)(g >> 1);
+            if (u > 0 && !mbar_wait_or_stop(bar + BAR_B_FREE + b, (u - 1u) & 1u, s_stop)) return false;   // product g - 2 has read the buffer
+            if (warp < 4) {
+                // the drain of item g - 2 has read its flip words (every warp reads them before it frees the accumulator)
+                if (u > 0 && !mbar_wait_or_stop(bar + BAR_ACC_FREE + b, (u - 1u) & 1u, s_stop)) return false;
+                const uint32_t row = (uint32_t)tid;   // 0..127
+                const uint4 w = rng_words(p.rng, p.id0 + (uint32_t)c_stage.n, 0u, (uint32_t)(c_stage.tile_base >> 7) + row);
+                reinterpret_cast<uint4*>(smem + kOffFlips + b * 2048u)[row] = w;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar + BAR_FLIPS + b);
+            }
+            hbutterfly(pre[0], pre[1]);   // column bit 5
+            hbutterfly(pre[2], pre[3]);
+            hbutterfly(pre[0], pre[2]);   // column bit 6
+            hbutterfly(pre[1], pre[3]);
+            unsigned char* const dst = smem + kOffB + b * kBBytes + sq * kBGroupStride + (srow >> 3) * 128u + (srow & 7u) * 16u;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) *reinterpret_cast<uint4*>(dst + 4 * t * kBGroupStride) = pre[t];
+            fence_generic_before_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar + BAR_B_FULL + b);
+            advance(c_stage);
+            return true;
+        };
+        // drain item g: accumulator -> registers, H_32 over the 32 columns, flip, add
+        auto drain_item = [&](int64_t g) -> bool {
+            const uint32_t b = (uint32_t)g & 1u, u = (uint32_t)(g >> 1);
+            const int n = c_drain.n;
+            const int64_t tile_base = c_drain.tile_base;
+            advance(c_drain);
+            if (!mbar_wait_or_stop(bar + BAR_ACC_FULL + b, u & 1u, s_stop)) return false;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            float v[32];
+            tmem_load32(tmem_base + ((lq * 32u) << 16) + b * 128u + cw * 32u, v);
+            if (!mbar_wait_or_stop(bar + BAR_FLIPS + b, u & 1u, s_stop)) return false;
+            const uint32_t fw = reinterpret_cast<const uint32_t*>(smem + kOffFlips + b * 2048u)[jrow * 4u + cw];
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar + BAR_ACC_FREE + b);
+            butterflies32<31>(v);
+            if (p.amp_mode == AMP_WEIGHT) {
+                const float wamp = amplitude_at(p, n, tile_base);
+#pragma unroll
+                for (int r = 0; r < 32; ++r) accv[r] = fmaf(flip_by_bit(v[r], fw, r), wamp, accv[r]);
+            } else {
+#pragma unroll
+                for (int r = 0; r < 32; ++r) accv[r] += flip_by_bit(v[r], fw, r);
+            }
+            if (n == W - 1) {
+                // the tile's sum is complete: scale and store 32 consecutive coordinates
+                const int64_t i0 = tile_base + jrow * 128u + cw * 32u;
+                const float sc = p.scale * (p.amp_mode == AMP_SCALE ? amplitude_at(p, 0, tile_base) : 1.f);
+                float* const dst = static_cast<float*>(p.dst) + i0;
+                if (i0 + 32 <= p.d_out) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        float4 o = make_float4(accv[4 * q], accv[4 * q + 1], accv[4 * q + 2], accv[4 * q + 3]);
+                        float4* const d4 = reinterpret_cast<float4*>(dst) + q;
+                        if (p.overwrite == 2) {
+                            const float4 c = *d4;
+                            o = make_float4(fmaf(o.x, sc, c.x), fmaf(o.y, sc, c.y), fmaf(o.z, sc, c.z), fmaf(o.w, sc, c.w));
+                        } else {
+                            if (!p.overwrite) {
+                                const float4 c = *d4;
+                                o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
+                            }
+                            o.x *= sc; o.y *= sc; o.z *= sc; o.w *= sc;
+                        }
+                        *d4 = o;
+                    }
+                } else {
+#pragma unroll
+                    for (int r = 0; r < 32; ++r) {
+                        if (i0 + r < p.d_out) {
+                            float o = accv[r];
+                            if (p.overwrite == 2) {
+                                dst[r] = fmaf(o, sc, dst[r]);
+                            } else {
+                                if (!p.overwrite) o += dst[r];
+                                dst[r] = o * sc;
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int r = 0; r < 32; ++r) accv[r] = 0.f;
+            }
+            return true;
+        };
+
+#pragma unroll
+        for (int r = 0; r < 32; ++r) accv[r] = 0.f;
+        if (nitems > 0) load_item();
+        for (int64_t g = 0; g < nitems && ok; ++g) {
+            ok = stage_item(g);
+            if (!ok) break;
+            if (g + 1 < nitems) load_item();          // in flight underneath the drain below
+            if (g > 0) ok = drain_item(g - 1);
+        }
+        if (ok && nitems > 0) ok = drain_item(nitems - 1);
+        if (!ok && lane == 0 && atomicExch((int*)s_stop, 1) == 0) atomicAdd(&g_tcrow_wait_timeouts, 1);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == kWorkerWarps) {
+        __syncwarp();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+    }
+}
+
+// one packed plane's fp16 intermediate, contiguous tiles of 2^14, whole tiles only
+bool tc_row_applicable(const PassParams& p, int T) { return T == kT && p.P == 1 && (p.dp >> kT) >= 1 && (p.dp >> kT) <= 0x7FFFFFFF; }
+
+cudaError_t launch_tc_row(const PassParams& p, cudaStream_t s)
+{
+    cudaError_t e = cudaFuncSetAttribute(tc_row_final_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const int64_t ntiles = p.dp >> kT;
+    const int64_t blocks = ntiles < sms ? ntiles : sms;
+    tc_row_final_kernel<<<(unsigned)blocks, kThreads, kSmemBytes, s>>>(p, (int)ntiles);
+    return cudaGetLastError();
+}
+
+cudaError_t tcrow_timeouts(int* out) { return cudaMemcpyFromSymbol(out, g_tcrow_wait_timeouts, sizeof(int)); }
+
+}  // namespace fosgd

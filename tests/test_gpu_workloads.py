@@ -323,18 +323,98 @@ def test_tensor_core_pass_matches_plain_alu_pass(F, cfg, block_log2):
     lam = 0.37
     ws = torch.empty(F.workspace_bytes(F.OP_AGGREGATE, d, block_log2=block_log2) * M, dtype=torch.uint8, device=DEV)
     acc = {}
-    for on in (False, True):
-        prev = F.set_tensor_core_pass(on)
+    for mask in (0, F.TC_STRIDED, F.TC_CONTIGUOUS, F.TC_STRIDED | F.TC_CONTIGUOUS):
+        prev = F.set_tensor_core_pass(mask)
         try:
             a = torch.empty(dp, dtype=torch.float32, device=DEV)
             F.server_aggregate(bits, d, a, lam, seed, step, block_log2=block_log2, ws=ws)
             torch.cuda.synchronize()
-            acc[on] = a
+            acc[mask] = a
         finally:
             F.set_tensor_core_pass(prev)
-    assert torch.equal(acc[True], acc[False])
+    for mask in acc:
+        assert torch.equal(acc[mask], acc[0]), mask
     gbar = np.zeros(dp)
     for part in pmap(lambda n: oracle.decode_full(words[n], d, seed, step, n, lam, block_log2=block_log2), range(M)):
         gbar += part
-    assert_l2_close(acc[True].cpu().numpy(), gbar / M)
+    assert_l2_close(acc[F.TC_CONTIGUOUS].cpu().numpy(), gbar / M)
     assert F.async_timeouts() == 0
+
+
+def test_tensor_core_contiguous_pass_sinks(F):
+    """The contiguous decode pass on the tensor cores (H_128 as an fp16 product, the other seven stages on the
+    plain ALUs) in every form of its sink: a decoder that returns d < d' coordinates, chunked aggregation
+    (begin / add / end), per-worker amplitudes read on the device, and the update x <- x - step * D(q): each bit
+    for bit against the plain-ALU pass (all values are exact integers until the final scale), the first also
+    against the oracle."""
+    d, seed, step, M = (1 << 24) - 70_001, 17, 4, 3
+    dp = F.padded_dim(d)
+    rng = np.random.default_rng(3)
+    words = rng.integers(0, 2 ** 32, (M, dp // 32), dtype=np.uint64).astype(np.uint32)
+    bits = torch.from_numpy(words.view(np.int32)).to(DEV)
+    ws = torch.empty(F.workspace_bytes(F.OP_AGGREGATE, d) * 2, dtype=torch.uint8, device=DEV)
+    lam, lam_s = 0.21, 1.7
+    amp = torch.tensor([[0.5], [1.25], [3.0]], dtype=torch.float32, device=DEV)   # one block of 2^24 per worker
+    amp_s = torch.tensor([0.75], dtype=torch.float32, device=DEV)
+    x0 = torch.randn(d, generator=torch.Generator(device=DEV).manual_seed(1), device=DEV)
+    res = {}
+    for mask in (0, F.TC_CONTIGUOUS):
+        prev = F.set_tensor_core_pass(mask)
+        try:
+            one = torch.full((d + 64,), 7.0, dtype=torch.float32, device=DEV)
+            F.decode(bits[1], d, one, lam, seed, step, 1, ws=ws)
+            acc = torch.empty(dp, dtype=torch.float32, device=DEV)
+            F.server_aggregate(bits[:2], d, acc, lam, seed, step, N_total=M, flags=F.AGG_BEGIN, ws=ws)
+            F.server_aggregate(bits[2:], d, acc, lam, seed, step, N_total=M, worker_id0=2, flags=F.AGG_END, ws=ws)
+            accw = torch.empty(dp, dtype=torch.float32, device=DEV)
+            F.server_aggregate_dev(bits, d, accw, amp, seed, step, lam_s=amp_s, block_log2=24, per_block=True, ws=ws)
+            x = x0.clone()
+            F.downlink_apply(bits[0], d, x, lam_s, seed, step, 0.125, ws=ws)
+            torch.cuda.synchronize()
+            res[mask] = (one, acc, accw, x)
+        finally:
+            F.set_tensor_core_pass(prev)
+    for a, b in zip(res[0], res[F.TC_CONTIGUOUS]):
+        assert torch.equal(a, b)
+    one = res[F.TC_CONTIGUOUS][0]
+    assert bool((one[d:] == 7.0).all())                       # nothing written beyond the d outputs
+    assert_l2_close(one[:d].cpu().numpy(), oracle.decode_full(words[1], d, seed, step, 1, lam)[:d])
+    assert F.async_timeouts() == 0
+
+
+@pytest.mark.parametrize("d,M,ws_workers,extra", [
+    (1 << 24, 3, 3, True),                 # one launch, progress words behind the intermediates
+    (1 << 24, 3, 3, False),                # scratch for exactly three workers: launches of two and one
+    ((1 << 24) - 70_001, 5, 2, True),      # ragged length (a partial last row of the strided view), three launches
+    ((1 << 23) + 5, 2, 2, True),           # mostly padding
+])
+def test_fused_encoder_matches_two_kernel_encoder(F, d, M, ws_workers, extra):
+    """The one-kernel uplink encoder of a 2^24-long transform (strided and contiguous pass side by side in
+    every block) against the oracle on one worker, and word for word against the same encoder run as two
+    kernels."""
+    seed, step = 5, 9
+    dp = F.padded_dim(d)
+    assert dp == 1 << 24
+    stride = (d + 7) // 8 * 8
+    g = torch.Generator(device=DEV).manual_seed(d % 1000 + M)
+    grads = torch.randn(M, stride, generator=g, device=DEV) * torch.rand(M, 1, generator=g, device=DEV)
+    lam = F.lambda_(float(grads[:, :d].double().norm(dim=1).max()), 2.0, dp)
+    nbytes = F.workspace_bytes(F.OP_ENCODE, d) * ws_workers + (F.fused_sync_bytes(ws_workers) if extra else 0)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=DEV)
+    out = {}
+    for on in (True, False):
+        prev = F.set_fused_encoder(on)
+        try:
+            bits = torch.zeros(M, dp // 32, dtype=torch.int32, device=DEV)
+            with F.PassTrace() as tr:
+                F.encode(grads, d, bits, lam, seed, step, ws=ws, worker_stride=stride, worker_id0=2)
+            torch.cuda.synchronize()
+            assert any(lab.startswith("fused") for lab in tr.labels) == on, tr.labels
+            out[on] = bits
+        finally:
+            F.set_fused_encoder(prev)
+    assert torch.equal(out[True], out[False])
+    assert F.async_timeouts() == 0
+    n = M - 1
+    ref, margin = oracle.encode(grads[n, :d].cpu().double().numpy(), seed, step, 2 + n, lam, want_margin=True)
+    assert_bits_match(to_np_words(out[True][n])[None], ref, margin, lam)
