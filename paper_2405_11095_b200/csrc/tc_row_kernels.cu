@@ -16,11 +16,14 @@
 // All values are integers below 2^24 in magnitude, so the result equals the plain-ALU kernel's bit
 // for bit.
 //
-// A block is 16 worker warps and one warp that issues the products.  It keeps a tile position and
-// walks the workers (sums in registers), then moves to its next tile.  Per item (tile, worker) a
-// worker warp stages its share of Z into one of two operand buffers, then drains the accumulator of
-// the previous item while the product of this one runs.  Synchronisation is by mbarriers only
-// (operand full / free, accumulator full / free, flips ready); every wait is bounded.
+// A block is 16 worker warps, one warp that issues the products and one service warp.  It keeps a tile
+// position and walks the workers (sums in registers), then moves to its next tile.  The service warp
+// keeps whole tiles (32 KiB, contiguous) arriving through the bulk copy engine into a ring of three
+// landing slots and makes the flip words of the items.  Per item (tile, worker) a worker warp turns its
+// share of a landed tile into the operand layout in one of two operand buffers, then drains the
+// accumulator of the previous item while the product of this one runs.  Synchronisation is by
+// mbarriers only (slot landed / read, operand full / free, accumulator full / free, flips ready);
+// every wait is bounded.
 #include "common.cuh"
 
 namespace fosgd {
@@ -31,7 +34,10 @@ namespace {
 
 constexpr int kT = 14;
 constexpr int kWorkerWarps = 16;
-constexpr int kThreads = (kWorkerWarps + 1) * 32;
+constexpr int kIssueWarp = kWorkerWarps, kServiceWarp = kWorkerWarps + 1;
+constexpr int kThreads = (kWorkerWarps + 2) * 32;
+constexpr int kRing = 3;                                   // landing slots for whole tiles (bulk copies in flight)
+constexpr uint32_t kTileBytes = 2u << kT;                  // one fp16 tile
 constexpr uint32_t kAChunkStride = 128;                    // bytes between core matrices along K
 constexpr uint32_t kAGroupStride = 16 * 128;               // bytes between groups of eight rows of A
 constexpr uint32_t kBGroupStride = 16 * 128 + 32;          // bytes between groups of eight columns of B (+32: staging stores hit distinct banks)
@@ -39,10 +45,12 @@ constexpr uint32_t kOffA = 0;                              // H_128 as fp16: 32 
 constexpr uint32_t kOffB = 32768;                          // two operand buffers
 constexpr uint32_t kBBytes = 16 * kBGroupStride;
 constexpr uint32_t kOffFlips = kOffB + 2 * kBBytes;        // two buffers of 128 rows x 4 flip words
-constexpr uint32_t kOffBar = kOffFlips + 2 * 2048;         // ten mbarriers, stop word, tensor-memory base
-constexpr uint32_t kSmemBytes = kOffBar + 128;
+constexpr uint32_t kOffLand = kOffFlips + 2 * 2048;        // kRing landing slots
+constexpr uint32_t kOffBar = kOffLand + kRing * kTileBytes;   // mbarriers, stop word, tensor-memory base
+constexpr int kNumBars = 10 + 2 * kRing;
+constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16;
 
-enum { BAR_B_FULL = 0, BAR_B_FREE = 2, BAR_ACC_FULL = 4, BAR_ACC_FREE = 6, BAR_FLIPS = 8 };
+enum { BAR_B_FULL = 0, BAR_B_FREE = 2, BAR_ACC_FULL = 4, BAR_ACC_FREE = 6, BAR_FLIPS = 8, BAR_LAND_FULL = 10, BAR_LAND_FREE = 10 + kRing };
 
 // instruction descriptor: D = f32 (1 << 4), A = B = fp16 (0), A K-major, B MN-major (1 << 16), N = 128, M = 128
 constexpr uint32_t kIdescF16 = (1u << 4) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
@@ -86,10 +94,10 @@ __device__ __forceinline__ bool mbar_wait_or_stop(uint64_t* bar, uint32_t parity
     return false;
 }
 
-// 32 consecutive accumulator columns of this thread's lane
-__device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&v)[32])
+// 32 consecutive accumulator columns of this thread's lane: the load is asynchronous; the registers may be
+// read after tmem_load32_wait, which names them so that no use can be scheduled before it.
+__device__ __forceinline__ void tmem_load32_issue(uint32_t taddr, uint32_t (&u)[32])
 {
-    uint32_t u[32];
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -99,9 +107,16 @@ __device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&v)[32])
           "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
           "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
         : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int r = 0; r < 32; ++r) v[r] = __uint_as_float(u[r]);
+}
+
+__device__ __forceinline__ void tmem_load32_wait(uint32_t (&u)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]),
+                   "+r"(u[8]), "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15]),
+                   "+r"(u[16]), "+r"(u[17]), "+r"(u[18]), "+r"(u[19]), "+r"(u[20]), "+r"(u[21]), "+r"(u[22]), "+r"(u[23]),
+                   "+r"(u[24]), "+r"(u[25]), "+r"(u[26]), "+r"(u[27]), "+r"(u[28]), "+r"(u[29]), "+r"(u[30]), "+r"(u[31])
+                 :: "memory");
 }
 
 __device__ __forceinline__ void hbutterfly(uint4& a, uint4& b)
@@ -125,8 +140,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
     const int warp = tid >> 5;
     const uint32_t lane = tid & 31;
     uint64_t* const bar = reinterpret_cast<uint64_t*>(smem + kOffBar);
-    volatile int* const s_stop = reinterpret_cast<volatile int*>(smem + kOffBar + 96);
-    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 100);
+    volatile int* const s_stop = reinterpret_cast<volatile int*>(smem + kOffBar + kNumBars * 8);
+    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + kNumBars * 8 + 4);
 
     // ---- once per block: the constant operand, barriers, tensor memory ----
     if (tid < 512) {
@@ -146,7 +161,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
                 make_uint4(w[0], w[1], w[2], w[3]);
         }
     }
-    if (warp == kWorkerWarps) {
+    if (warp == kIssueWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -157,7 +172,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
             mbar_init(bar + BAR_B_FREE + b, 1);
             mbar_init(bar + BAR_ACC_FULL + b, 1);
             mbar_init(bar + BAR_ACC_FREE + b, kWorkerWarps);
-            mbar_init(bar + BAR_FLIPS + b, 4);
+            mbar_init(bar + BAR_FLIPS + b, 1);
+        }
+#pragma unroll
+        for (int r = 0; r < kRing; ++r) {
+            mbar_init(bar + BAR_LAND_FULL + r, 1);
+            mbar_init(bar + BAR_LAND_FREE + r, kWorkerWarps);
         }
         *s_stop = 0;
     }
@@ -169,9 +189,23 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
 
     const int W = p.nworkers;
     const int my_tiles = ((int)blockIdx.x < ntiles) ? (ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-    const int64_t nitems = (int64_t)my_tiles * W;   // item g: tile blockIdx.x + (g / W) * gridDim.x, worker g % W
+    const int64_t nitems = (int64_t)my_tiles * W;   // item g: this block's tile number g / W, worker g % W
 
-    if (warp == kWorkerWarps) {
+    // where an item sits: first coordinate of its tile and its worker; advanced item by item (worker fastest)
+    struct Cursor {
+        int64_t tile_base;
+        int n;
+    };
+    const int64_t tile_step = (int64_t)gridDim.x << kT;
+    auto advance = [&](Cursor& c) {
+        if (++c.n == W) {
+            c.n = 0;
+            c.tile_base += tile_step;
+        }
+    };
+    const Cursor c_first{(int64_t)blockIdx.x << kT, 0};
+
+    if (warp == kIssueWarp) {
         // ================= the warp that issues the products =================
         if (lane == 0) {
             const uint64_t adesc = umma_desc(smem_u32(smem + kOffA), kAChunkStride, kAGroupStride);
@@ -196,58 +230,86 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
                 for (int64_t h = (g >= 2 ? g - 2 : 0); h < g; ++h) mbar_wait(bar + BAR_ACC_FULL + (h & 1), (uint32_t)(h >> 1) & 1u);
             }
         }
+    } else if (warp == kServiceWarp) {
+        // ================= the service warp: tiles in through the copy engine, flip words =================
+        // Lane 0 keeps kRing bulk copies of whole tiles (32 KiB, contiguous) in flight; all lanes make the
+        // flip words of the items (four generator calls per lane: 128 rows x 128 flips).
+        Cursor c_ld = c_first, c_fl = c_first;
+        bool ok = true;
+        int64_t issued = 0;   // lane 0: copies started
+        auto issue_load = [&](int64_t g) -> bool {
+            const uint32_t r = (uint32_t)(g % kRing), u = (uint32_t)(g / kRing);
+            if (u > 0 && !mbar_wait_or_stop(bar + BAR_LAND_FREE + r, (u - 1u) & 1u, s_stop)) return false;   // every warp has read the slot
+            const __half* const src = static_cast<const __half*>(p.src) + (int64_t)c_ld.n * p.src_stride + c_ld.tile_base;
+            advance(c_ld);
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar + BAR_LAND_FULL + r)), "r"(kTileBytes) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_u32(smem + kOffLand + r * kTileBytes)), "l"(src), "r"(kTileBytes), "r"(smem_u32(bar + BAR_LAND_FULL + r)) : "memory");
+            ++issued;
+            return true;
+        };
+        if (lane == 0) {
+            for (int64_t g = 0; g < kRing - 1 && g < nitems && ok; ++g) ok = issue_load(g);
+        }
+        for (int64_t g = 0; g < nitems; ++g) {
+            if (lane == 0 && ok && g + kRing - 1 < nitems) ok = issue_load(g + kRing - 1);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            const uint32_t b = (uint32_t)g & 1u, u = (uint32_t)(g >> 1);
+            // the drain of item g - 2 has read its flip words (every warp reads them before it frees the accumulator)
+            if (u > 0 && !mbar_wait_or_stop(bar + BAR_ACC_FREE + b, (u - 1u) & 1u, s_stop)) { ok = false; }
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            const uint32_t id = p.id0 + (uint32_t)c_fl.n, c0 = (uint32_t)(c_fl.tile_base >> 7);
+            advance(c_fl);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t row = lane + 32u * k;
+                reinterpret_cast<uint4*>(smem + kOffFlips + b * 2048u)[row] = rng_words(p.rng, id, 0u, c0 + row);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar + BAR_FLIPS + b);
+        }
+        if (!ok && lane == 0) {
+            if (atomicExch((int*)s_stop, 1) == 0) atomicAdd(&g_tcrow_wait_timeouts, 1);
+        }
+        // copies started but possibly not landed yet: one more bounded wait each, so that the engine is not
+        // left writing into shared memory that the next block of this SM may own
+        if (lane == 0) {
+            for (int64_t h = (issued >= kRing ? issued - kRing : 0); h < issued; ++h)
+                mbar_wait(bar + BAR_LAND_FULL + (h % kRing), (uint32_t)(h / kRing) & 1u);
+        }
     } else {
         // ================= worker warps: stage, drain, flip, sum =================
         const uint32_t srow = (uint32_t)tid >> 2, sq = (uint32_t)tid & 3u;       // staging role: row of the tile, column chunks sq + 4 t
         const uint32_t lq = (uint32_t)warp & 3u, cw = (uint32_t)warp >> 2;       // drain role: lane quarter, 32 of the 128 columns
         const uint32_t jrow = lq * 32u + lane;                                  // output row (index bits 7..13)
         float accv[32];
-        uint4 pre[4];
         bool ok = true;
+        Cursor c_drain = c_first;
 
-        // where an item sits: first coordinate of its tile and its worker; advanced item by item (worker fastest)
-        struct Cursor {
-            int64_t tile_base;
-            int n;
-        };
-        const int64_t tile_step = (int64_t)gridDim.x << kT;
-        auto advance = [&](Cursor& c) {
-            if (++c.n == W) {
-                c.n = 0;
-                c.tile_base += tile_step;
-            }
-        };
-        Cursor c_load{(int64_t)blockIdx.x << kT, 0}, c_stage = c_load, c_drain = c_load;
-        auto load_item = [&]() {
-            const __half* const src = static_cast<const __half*>(p.src) + (int64_t)c_load.n * p.src_stride + c_load.tile_base + srow * 128u + sq * 8u;
-#pragma unroll
-            for (int t = 0; t < 4; ++t) pre[t] = __ldcs(reinterpret_cast<const uint4*>(src + 32 * t));
-            advance(c_load);
-        };
-        // stage item g from `pre` into its operand buffer (and, warps 0..3, its flip words)
+        // stage item g: landed tile -> H_4 over column bits 5, 6 -> operand buffer
         auto stage_item = [&](int64_t g) -> bool {
             const uint32_t b = (uint32_t)g & 1u, u = (uint32_t)(g >> 1);
-            if (u > 0 && !mbar_wait_or_stop(bar + BAR_B_FREE + b, (u - 1u) & 1u, s_stop)) return false;   // product g - 2 has read the buffer
-            if (warp < 4) {
-                // the drain of item g - 2 has read its flip words (every warp reads them before it frees the accumulator)
-                if (u > 0 && !mbar_wait_or_stop(bar + BAR_ACC_FREE + b, (u - 1u) & 1u, s_stop)) return false;
-                const uint32_t row = (uint32_t)tid;   // 0..127
-                const uint4 w = rng_words(p.rng, p.id0 + (uint32_t)c_stage.n, 0u, (uint32_t)(c_stage.tile_base >> 7) + row);
-                reinterpret_cast<uint4*>(smem + kOffFlips + b * 2048u)[row] = w;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar + BAR_FLIPS + b);
-            }
+            const uint32_t r = (uint32_t)(g % kRing), ur = (uint32_t)(g / kRing);
+            if (!mbar_wait_or_stop(bar + BAR_LAND_FULL + r, ur & 1u, s_stop)) return false;               // the tile has landed
+            uint4 pre[4];
+            const unsigned char* const land = smem + kOffLand + r * kTileBytes + srow * 256u + sq * 16u;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) pre[t] = *reinterpret_cast<const uint4*>(land + 64 * t);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar + BAR_LAND_FREE + r);
             hbutterfly(pre[0], pre[1]);   // column bit 5
             hbutterfly(pre[2], pre[3]);
             hbutterfly(pre[0], pre[2]);   // column bit 6
             hbutterfly(pre[1], pre[3]);
+            if (u > 0 && !mbar_wait_or_stop(bar + BAR_B_FREE + b, (u - 1u) & 1u, s_stop)) return false;   // product g - 2 has read the buffer
             unsigned char* const dst = smem + kOffB + b * kBBytes + sq * kBGroupStride + (srow >> 3) * 128u + (srow & 7u) * 16u;
 #pragma unroll
             for (int t = 0; t < 4; ++t) *reinterpret_cast<uint4*>(dst + 4 * t * kBGroupStride) = pre[t];
             fence_generic_before_async();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar + BAR_B_FULL + b);
-            advance(c_stage);
             return true;
         };
         // drain item g: accumulator -> registers, H_32 over the 32 columns, flip, add
@@ -258,16 +320,23 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
             advance(c_drain);
             if (!mbar_wait_or_stop(bar + BAR_ACC_FULL + b, u & 1u, s_stop)) return false;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            float v[32];
-            tmem_load32(tmem_base + ((lq * 32u) << 16) + b * 128u + cw * 32u, v);
-            if (!mbar_wait_or_stop(bar + BAR_FLIPS + b, u & 1u, s_stop)) return false;
+            uint32_t raw[32];
+            tmem_load32_issue(tmem_base + ((lq * 32u) << 16) + b * 128u + cw * 32u, raw);
+            if (!mbar_wait_or_stop(bar + BAR_FLIPS + b, u & 1u, s_stop)) {
+                tmem_load32_wait(raw);
+                return false;
+            }
             const uint32_t fw = reinterpret_cast<const uint32_t*>(smem + kOffFlips + b * 2048u)[jrow * 4u + cw];
+            const float wamp = (p.amp_mode == AMP_WEIGHT) ? amplitude_at(p, n, tile_base) : 1.f;
+            tmem_load32_wait(raw);
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(bar + BAR_ACC_FREE + b);
+            float v[32];
+#pragma unroll
+            for (int r = 0; r < 32; ++r) v[r] = __uint_as_float(raw[r]);
             butterflies32<31>(v);
             if (p.amp_mode == AMP_WEIGHT) {
-                const float wamp = amplitude_at(p, n, tile_base);
 #pragma unroll
                 for (int r = 0; r < 32; ++r) accv[r] = fmaf(flip_by_bit(v[r], fw, r), wamp, accv[r]);
             } else {
@@ -318,19 +387,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
 
 #pragma unroll
         for (int r = 0; r < 32; ++r) accv[r] = 0.f;
-        if (nitems > 0) load_item();
         for (int64_t g = 0; g < nitems && ok; ++g) {
             ok = stage_item(g);
             if (!ok) break;
-            if (g + 1 < nitems) load_item();          // in flight underneath the drain below
-            if (g > 0) ok = drain_item(g - 1);
+            if (g > 0) ok = drain_item(g - 1);        // underneath the product of item g
         }
         if (ok && nitems > 0) ok = drain_item(nitems - 1);
         if (!ok && lane == 0 && atomicExch((int*)s_stop, 1) == 0) atomicAdd(&g_tcrow_wait_timeouts, 1);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == kWorkerWarps) {
+    if (warp == kIssueWarp) {
         __syncwarp();
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
