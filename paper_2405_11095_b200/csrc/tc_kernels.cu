@@ -22,10 +22,12 @@
 // 0x6400 + u = 1024 + u (exact for 0 <= u <= 1024): h = bits(0x6400 + D + 512) = 1536 + v / 2 and
 // v = 2 h - 3072 in one packed fused multiply-add; row 0 simply adds 0x6400 instead of 0x6600.
 //
-// Tensor memory: 512 columns = four 128-column accumulators, used as two pairs in turn: while the
-// threads drain one pair the products of the next pair run.  A block (1024 threads, one per SM,
-// persistent over tiles) prefetches the packed rows of its next tile under the epilogue; every
-// wait is bounded.
+// A block is 16 worker warps and one warp that issues the products, persistent over tiles.  Tensor
+// memory holds four 128-column accumulators used in turn, so that while the worker warps drain one
+// (tcgen05.ld, convert, 64 contiguous bytes per thread straight to global memory) the products of the
+// next ones run.  The packed rows of the next tile are fetched into registers under the current one.
+// Synchronisation is by mbarriers (operands staged / all products of the tile done, accumulator full /
+// drained); every wait is bounded.
 #include "common.cuh"
 
 namespace fosgd {
@@ -34,16 +36,20 @@ static __device__ int g_tc_wait_timeouts;   // blocks that abandoned a bounded w
 
 namespace {
 
-constexpr int kTcThreads = 1024;
+constexpr int kWorkerWarps = 16;
+constexpr int kWorkers = kWorkerWarps * 32;
+constexpr int kTcThreads = kWorkers + 32;
 constexpr uint32_t kBOperandBytes = 8 * 2064;                 // eight column groups of 16, 2048 B each + 16 B so that they sit on different banks
 constexpr uint32_t kOffA = 0;                                 // H_128 as int8, K-major core matrices: 16 KiB
 constexpr uint32_t kOffB = 16384;                             // eight B operands
 constexpr uint32_t kOffBits = kOffB + 8 * kBOperandBytes;     // the tile's packed rows: 1024 x 16 B
 constexpr uint32_t kOffLut = kOffBits + 16384;                // byte -> eight bytes of {0, 1}: 2 KiB
-constexpr uint32_t kOffBar = kOffLut + 2048;                  // two mbarriers, tensor-memory base address
-constexpr uint32_t kStagePitch = 272;                         // bytes per staged row: 128 fp16 + 16 (rows land on different banks)
-constexpr uint32_t kOffStage = kOffBar + 32;                  // one accumulator as fp16: 128 rows
-constexpr uint32_t kTcSmemBytes = kOffStage + 128 * kStagePitch;
+constexpr uint32_t kOffBar = kOffLut + 2048;                  // eleven mbarriers, stop word, tensor-memory base address
+constexpr uint32_t kPatchPitch = 80;                          // bytes per row of a warp's output patch: 32 fp16 + 16 (rows land on different banks)
+constexpr uint32_t kOffPatch = kOffBar + 128;                 // one patch of 32 rows per worker warp
+constexpr uint32_t kTcSmemBytes = kOffPatch + kWorkerWarps * 32 * kPatchPitch;
+
+enum { BAR_B_FULL = 0, BAR_B_DONE = 1, BAR_ACC_FULL = 2, BAR_ACC_FREE = 6, BAR_BITS = 10 };
 
 // shared-memory matrix descriptor, no swizzle: start address, leading and stride byte offsets in
 // units of 16 bytes, descriptor version 1
@@ -68,16 +74,42 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescI8), "r"(accumulate) : "memory");
 }
 
-// 16 consecutive accumulator columns of this thread's lane
-__device__ __forceinline__ void tmem_load16(uint32_t taddr, uint32_t (&v)[16])
+// 32 consecutive accumulator columns of this thread's lane
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t (&u)[32])
 {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+          "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
+          "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
+          "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
         : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]),
+                   "+r"(u[8]), "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15]),
+                   "+r"(u[16]), "+r"(u[17]), "+r"(u[18]), "+r"(u[19]), "+r"(u[20]), "+r"(u[21]), "+r"(u[22]), "+r"(u[23]),
+                   "+r"(u[24]), "+r"(u[25]), "+r"(u[26]), "+r"(u[27]), "+r"(u[28]), "+r"(u[29]), "+r"(u[30]), "+r"(u[31])
+                 :: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// bounded wait that also gives up when the block's stop word is raised
+__device__ __forceinline__ bool mbar_wait_or_stop(uint64_t* bar, uint32_t parity, const volatile int* stop)
+{
+    for (int it = 0; it < (1 << 22); ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (done) return true;
+        if ((it & 255) == 255 && *stop) return false;
+    }
+    return false;
 }
 
 }  // namespace
@@ -89,10 +121,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_col_kernel(const PassParams 
     const int warp = tid >> 5;
     const uint32_t lane = tid & 31;
     uint64_t* const bar = reinterpret_cast<uint64_t*>(smem + kOffBar);
-    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 16);
+    volatile int* const s_stop = reinterpret_cast<volatile int*>(smem + kOffBar + 96);
+    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 100);
     const uint2* const lut = reinterpret_cast<const uint2*>(smem + kOffLut);
 
-    // ---- once per block: expansion table, the constant operand, barrier, tensor memory ----
+    // ---- once per block: expansion table, the constant operand, barriers, tensor memory ----
     if (tid < 256) {
         uint32_t lo = 0, hi = 0;
 #pragma unroll
@@ -102,28 +135,38 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_col_kernel(const PassParams 
         }
         reinterpret_cast<uint2*>(smem + kOffLut)[tid] = make_uint2(lo, hi);
     }
-    {
-        // A[m][k] = (-1)^popcount(m & k): row m, sixteen k per thread; core matrix = 8 rows x 16 bytes
-        const uint32_t m = (uint32_t)tid >> 3, kc = (uint32_t)tid & 7u;
-        uint32_t w[4];
+    if (tid < kWorkers) {
+        // A[m][k] = (-1)^popcount(m & k): row m, 32 of its k per thread; core matrix = 8 rows x 16 bytes
+        const uint32_t m = (uint32_t)tid >> 2, kc0 = ((uint32_t)tid & 3u) * 2u;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            w[q] = 0;
+        for (int c = 0; c < 2; ++c) {
+            uint32_t w[4];
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const uint32_t k = kc * 16u + 4u * q + b;
-                w[q] |= ((__popc(m & k) & 1) ? 0xFFu : 0x01u) << (8 * b);
+            for (int q = 0; q < 4; ++q) {
+                w[q] = 0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const uint32_t k = (kc0 + c) * 16u + 4u * q + b;
+                    w[q] |= ((__popc(m & k) & 1) ? 0xFFu : 0x01u) << (8 * b);
+                }
             }
+            *reinterpret_cast<uint4*>(smem + kOffA + (m & 7u) * 16u + (m >> 3) * 1024u + (kc0 + c) * 128u) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        *reinterpret_cast<uint4*>(smem + kOffA + (m & 7u) * 16u + (m >> 3) * 1024u + kc * 128u) = make_uint4(w[0], w[1], w[2], w[3]);
     }
-    if (warp == 0) {
+    if (warp == kWorkerWarps) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (tid == 0) {
-        mbar_init(bar + 0, 1);
-        mbar_init(bar + 1, 1);
+        mbar_init(bar + BAR_B_FULL, kWorkerWarps);
+        mbar_init(bar + BAR_B_DONE, 1);
+        mbar_init(bar + BAR_BITS, kWorkerWarps);
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            mbar_init(bar + BAR_ACC_FULL + a, 1);
+            mbar_init(bar + BAR_ACC_FREE + a, kWorkerWarps);
+        }
+        *s_stop = 0;
     }
     fence_generic_before_async();   // the constant operand, for the tensor core's reads
     tc_fence_before_sync();
@@ -133,146 +176,161 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_col_kernel(const PassParams 
 
     const uint32_t step = 1u << p.lo_log;
     const int64_t total = ntiles * p.nworkers;
-    const uint32_t cg = (uint32_t)tid & 7u, k1 = (uint32_t)tid >> 3;   // producer role: 16 columns of row k1 (of every t)
-    const uint32_t lq = (uint32_t)warp & 3u, cw = (uint32_t)warp >> 2; // epilogue role: lane quarter, 16 of an accumulator's 128 columns
-    const uint32_t j1 = lq * 32u + lane;                              // output row inside the 128-block
-    const uint32_t half_bits = (j1 == 0) ? 0x6400u : 0x6600u;          // fp16 pattern base: 1024 (+ 512 except on the offset row)
-    uint32_t commits[2] = {0, 0};
-    bool failed = false;
+    const int64_t nitems = ((int64_t)blockIdx.x < total) ? (total - (int64_t)blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
-    auto tile_origin = [&](int64_t item, int& n, uint32_t& i_tile) {
-        n = (int)(item / ntiles);
-        const uint32_t tile = (uint32_t)(item % ntiles);
-        const uint32_t col0 = (tile << 7) & (step - 1u);
-        const uint32_t hi = (tile << 7) >> p.lo_log;
-        i_tile = (hi << (p.lo_log + 10)) + col0;                      // row 0, column 0 of the tile
-    };
-    auto load_bits = [&](int64_t item) -> uint4 {
-        int n;
-        uint32_t i_tile;
-        tile_origin(item, n, i_tile);
-        const uint32_t* const bits = static_cast<const uint32_t*>(p.src) + (int64_t)n * p.src_stride;
-        return __ldg(reinterpret_cast<const uint4*>(bits + ((i_tile + (uint32_t)tid * step) >> 5)));
-    };
-    // four products (two accumulators) of pair `pr` (t' = 2 pr, 2 pr + 1) into columns (pr & 1) * 256 ...
-    auto issue_pair = [&](int pr) {
-        tc_fence_after_sync();
-        const uint64_t adesc = umma_desc(smem_u32(smem + kOffA), 128u, 1024u);
+    if (warp == kWorkerWarps) {
+        // ================= the warp that issues the products =================
+        if (lane == 0) {
+            const uint64_t adesc = umma_desc(smem_u32(smem + kOffA), 128u, 1024u);
+            bool ok = true;
+            int64_t issued = 0;   // products committed so far (eight per tile)
+            for (int64_t g = 0; g < nitems && ok; ++g) {
+                ok = mbar_wait_or_stop(bar + BAR_B_FULL, (uint32_t)g & 1u, s_stop);                 // the tile's eight operands are staged
+                for (int t = 0; t < 8 && ok; ++t) {
+                    const uint32_t a = (uint32_t)t & 3u, u = (uint32_t)(2 * g) + ((uint32_t)t >> 2);   // accumulator and how often it has been used
+                    if (u > 0) ok = mbar_wait_or_stop(bar + BAR_ACC_FREE + a, (u - 1u) & 1u, s_stop);   // drained
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint64_t bdesc = umma_desc(smem_u32(smem + kOffB + (uint32_t)t * kBOperandBytes), 128u, 2064u);
 #pragma unroll
-        for (int a = 0; a < 2; ++a) {
-            const uint64_t bdesc = umma_desc(smem_u32(smem + kOffB + (uint32_t)(2 * pr + a) * kBOperandBytes), 128u, 2064u);
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)   // K = 32 per instruction: two core matrices of A, four k-groups of B
-                umma_i8(tmem_base + (uint32_t)(pr & 1) * 256u + (uint32_t)a * 128u, adesc + (uint64_t)(ks * (256 >> 4)),
-                        bdesc + (uint64_t)(ks * (512 >> 4)), ks > 0 ? 1u : 0u);
-        }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar + (pr & 1))) : "memory");
-    };
-
-    uint4 next_bits = make_uint4(0, 0, 0, 0);
-    if ((int64_t)blockIdx.x < total) next_bits = load_bits(blockIdx.x);
-    for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
-        int n;
-        uint32_t i_tile;
-        tile_origin(item, n, i_tile);
-        // ---- the tile's packed rows into shared memory (16 bytes per row), the next tile's into registers ----
-        reinterpret_cast<uint4*>(smem + kOffBits)[tid] = next_bits;
-        __syncthreads();
-        if (item + gridDim.x < total) next_bits = load_bits(item + gridDim.x);
-        // ---- expand to bytes, H_8 over t on packed bytes, store the eight B operands ----
-        {
-            uint32_t x[8][4];
-#pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const uint32_t h = *reinterpret_cast<const uint16_t*>(smem + kOffBits + ((uint32_t)t * 128u + k1) * 16u + cg * 2u);
-                const uint2 a = lut[h & 0xFFu], b = lut[h >> 8];
-                x[t][0] = a.x; x[t][1] = a.y; x[t][2] = b.x; x[t][3] = b.y;
+                    for (int ks = 0; ks < 4; ++ks)   // K = 32 per instruction: two core matrices of A, four k-groups of B
+                        umma_i8(tmem_base + a * 128u, adesc + (uint64_t)(ks * (256 >> 4)), bdesc + (uint64_t)(ks * (512 >> 4)), ks > 0 ? 1u : 0u);
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar + BAR_ACC_FULL + a)) : "memory");
+                    ++issued;
+                }
+                if (ok) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar + BAR_B_DONE)) : "memory");
             }
+            if (!ok) {
+                if (atomicExch((int*)s_stop, 1) == 0) atomicAdd(&g_tc_wait_timeouts, 1);
+                // products already committed may still be running: one more bounded wait each before the tensor memory goes back
+                for (int64_t h = (issued >= 4 ? issued - 4 : 0); h < issued; ++h)
+                    mbar_wait(bar + BAR_ACC_FULL + (h & 3), (uint32_t)(h >> 2) & 1u);
+            }
+        }
+    } else {
+        // ================= worker warps: expand, H_8 on packed bytes, stage; drain and store =================
+        const uint32_t cg = (uint32_t)tid & 7u, k1 = (uint32_t)tid >> 3;     // staging role: 16 columns of rows k1 and k1 + 64 (of every t)
+        const uint32_t lq = (uint32_t)warp & 3u, cw = (uint32_t)warp >> 2;   // drain role: lane quarter, 32 of an accumulator's 128 columns
+        const uint32_t j1 = lq * 32u + lane;                                // output row inside the 128-block
+        const uint32_t half_bits = (j1 == 0) ? 0x6400u : 0x6600u;            // fp16 pattern base: 1024 (+ 512 except on the offset row)
+        unsigned char* const patch = smem + kOffPatch + (uint32_t)warp * 32u * kPatchPitch;
+        bool ok = true;
+
+        auto tile_origin = [&](int64_t item, int& n, uint32_t& i_tile) {
+            n = (int)(item / ntiles);
+            const uint32_t tile = (uint32_t)(item % ntiles);
+            const uint32_t col0 = (tile << 7) & (step - 1u);
+            const uint32_t hi = (tile << 7) >> p.lo_log;
+            i_tile = (hi << (p.lo_log + 10)) + col0;                        // row 0, column 0 of the tile
+        };
+        // this thread's two packed rows (tid and tid + 512) of an item: 16 bytes = 128 columns each
+        auto load_bits = [&](int64_t item, uint4 (&w)[2]) {
+            int n;
+            uint32_t i_tile;
+            tile_origin(item, n, i_tile);
+            const uint32_t* const bits = static_cast<const uint32_t*>(p.src) + (int64_t)n * p.src_stride;
 #pragma unroll
-            for (int s = 0; s < 3; ++s) {
-                const uint32_t bias = 0x01010101u << s;
+            for (int k = 0; k < 2; ++k) w[k] = __ldg(reinterpret_cast<const uint4*>(bits + ((i_tile + ((uint32_t)tid + 512u * k) * step) >> 5)));
+        };
+
+        uint4 next_bits[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+        if (nitems > 0) load_bits(blockIdx.x, next_bits);
+        for (int64_t g = 0; g < nitems && ok; ++g) {
+            const int64_t item = (int64_t)blockIdx.x + g * gridDim.x;
+            int n;
+            uint32_t i_tile;
+            tile_origin(item, n, i_tile);
+            // ---- the tile's packed rows into shared memory, the next tile's into registers ----
+            // (every worker has left the previous tile's rows behind: it passed that tile's first accumulator wait,
+            // which follows the arrival of all sixteen warps on the operand barrier)
+            reinterpret_cast<uint4*>(smem + kOffBits)[tid] = next_bits[0];
+            reinterpret_cast<uint4*>(smem + kOffBits)[tid + 512] = next_bits[1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar + BAR_BITS);
+            if (!mbar_wait_or_stop(bar + BAR_BITS, (uint32_t)g & 1u, s_stop)) { ok = false; break; }   // all sixteen warps' rows are in
+            if (g + 1 < nitems) load_bits(item + gridDim.x, next_bits);
+            // all eight products of the previous tile have read the operands
+            if (g > 0 && !mbar_wait_or_stop(bar + BAR_B_DONE, (uint32_t)(g - 1) & 1u, s_stop)) { ok = false; break; }
+            // ---- expand to bytes, H_8 over t on packed bytes, store the eight B operands ----
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t kr = k1 + 64u * (uint32_t)h;
+                uint32_t x[8][4];
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
-                    if (!(t & (1 << s))) {
+                    const uint32_t hw = *reinterpret_cast<const uint16_t*>(smem + kOffBits + ((uint32_t)t * 128u + kr) * 16u + cg * 2u);
+                    const uint2 a = lut[hw & 0xFFu], b = lut[hw >> 8];
+                    x[t][0] = a.x; x[t][1] = a.y; x[t][2] = b.x; x[t][3] = b.y;
+                }
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const uint32_t a = x[t][q], b = x[t | (1 << s)][q];
-                            x[t][q] = a + b;
-                            x[t | (1 << s)][q] = a - b + bias;
+                for (int s = 0; s < 3; ++s) {
+                    const uint32_t bias = 0x01010101u << s;
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        if (!(t & (1 << s))) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const uint32_t a = x[t][q], b = x[t | (1 << s)][q];
+                                x[t][q] = a + b;
+                                x[t | (1 << s)][q] = a - b + bias;
+                            }
                         }
                     }
                 }
-            }
 #pragma unroll
-            for (int t = 0; t < 8; ++t)
-                *reinterpret_cast<uint4*>(smem + kOffB + (uint32_t)t * kBOperandBytes + cg * 2064u + (k1 >> 3) * 128u + (k1 & 7u) * 16u) =
-                    make_uint4(x[t][0], x[t][1], x[t][2], x[t][3]);
-        }
-        fence_generic_before_async();
-        tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0) {
-            issue_pair(0);
-            issue_pair(1);
-        }
+                for (int t = 0; t < 8; ++t)
+                    *reinterpret_cast<uint4*>(smem + kOffB + (uint32_t)t * kBOperandBytes + cg * 2064u + (kr >> 3) * 128u + (kr & 7u) * 16u) =
+                        make_uint4(x[t][0], x[t][1], x[t][2], x[t][3]);
+            }
+            fence_generic_before_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar + BAR_B_FULL);
 
-        __half* const dst = static_cast<__half*>(p.dst) + (int64_t)n * p.dst_stride;
+            // ---- drain the eight accumulators: fp16 through the warp's patch to global memory ----
+            __half* const dst = static_cast<__half*>(p.dst) + (int64_t)n * p.dst_stride + i_tile + cw * 32u;
 #pragma unroll 1
-        for (int pr = 0; pr < 4; ++pr) {
-            // bounded wait for the pair's products; the block agrees on the outcome
-            if (!__syncthreads_and(mbar_wait(bar + (pr & 1), commits[pr & 1] & 1u) ? 1 : 0)) {
-                failed = true;
-                break;
-            }
-            ++commits[pr & 1];
-            tc_fence_after_sync();
-#pragma unroll 1
-            for (int a = 0; a < 2; ++a) {
-                // ---- accumulator -> fp16 -> staging tile (row j1, 16 of its 128 columns per warp) ----
-                uint32_t v[16];
-                tmem_load16(tmem_base + ((lq * 32u) << 16) + (uint32_t)(pr & 1) * 256u + (uint32_t)a * 128u + cw * 16u, v);
+            for (int t = 0; t < 8; ++t) {
+                const uint32_t a = (uint32_t)t & 3u, u = (uint32_t)(2 * g) + ((uint32_t)t >> 2);
+                if (!mbar_wait_or_stop(bar + BAR_ACC_FULL + a, u & 1u, s_stop)) { ok = false; break; }
+                tc_fence_after_sync();
+                uint32_t v[32];
+                tmem_load32(tmem_base + ((lq * 32u) << 16) + a * 128u + cw * 32u, v);
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar + BAR_ACC_FREE + a);
                 const __half2 two = __floats2half2_rn(2.f, 2.f), off = __floats2half2_rn(-3072.f, -3072.f);
-                unsigned char* const srow = smem + kOffStage + j1 * kStagePitch + cw * 32u;
+                // through the warp's patch, so that a store instruction writes 64 contiguous bytes of eight rows
+                // instead of 16 bytes of thirty-two
 #pragma unroll
-                for (int g = 0; g < 2; ++g) {
+                for (int q4 = 0; q4 < 4; ++q4) {
                     uint32_t w[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        const uint32_t hb = __byte_perm(v[8 * g + 2 * q] + half_bits, v[8 * g + 2 * q + 1] + half_bits, 0x5410);
-                        const __half2 h = __hfma2(*reinterpret_cast<const __half2*>(&hb), two, off);
-                        w[q] = *reinterpret_cast<const uint32_t*>(&h);
+                        const uint32_t hb = __byte_perm(v[8 * q4 + 2 * q] + half_bits, v[8 * q4 + 2 * q + 1] + half_bits, 0x5410);
+                        const __half2 hh = __hfma2(*reinterpret_cast<const __half2*>(&hb), two, off);
+                        w[q] = *reinterpret_cast<const uint32_t*>(&hh);
                     }
-                    *reinterpret_cast<uint4*>(srow + g * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4*>(patch + lane * kPatchPitch + q4 * 16) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
-                __syncthreads();
-                // ---- staging tile -> global memory: a warp instruction writes two whole rows ----
-                {
-                    const uint32_t tq = (uint32_t)(2 * pr + a);                       // t' of this accumulator
+                __syncwarp();
 #pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-                        const uint32_t r = (uint32_t)warp * 4u + 2u * k + (lane >> 4);       // 32 warps x 4 rows
-                        const uint4 q = *reinterpret_cast<const uint4*>(smem + kOffStage + r * kStagePitch + (lane & 15u) * 16u);
-                        __stcg(reinterpret_cast<uint4*>(dst + i_tile + (tq * 128u + r) * step + (lane & 15u) * 8u), q);   // L2 only: read next by another kernel
-                    }
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t r = 8u * i + (lane >> 2), c = lane & 3u;
+                    const uint4 q = *reinterpret_cast<const uint4*>(patch + r * kPatchPitch + c * 16u);
+                    __stcg(reinterpret_cast<uint4*>(dst + (size_t)((uint32_t)t * 128u + lq * 32u + r) * step + c * 8u), q);   // L2 only: read next by another kernel
                 }
-                if (a == 0) __syncthreads();   // the staging tile is free again
+                __syncwarp();
             }
-            tc_fence_before_sync();
-            __syncthreads();   // this pair of accumulators (and the staging tile) may be reused
-            if (tid == 0 && pr + 2 < 4) issue_pair(pr + 2);
         }
-        if (failed) break;
+        if (!ok && lane == 0 && atomicExch((int*)s_stop, 1) == 0) atomicAdd(&g_tc_wait_timeouts, 1);
     }
-    if (failed) {
-        // products may still be running: one more bounded wait on both barriers before the tensor memory goes back
-        if (tid == 0) {
-            atomicAdd(&g_tc_wait_timeouts, 1);
-            mbar_wait(bar + 0, commits[0] & 1u);
-            mbar_wait(bar + 1, commits[1] & 1u);
-        }
-        __syncthreads();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kWorkerWarps) {
+        __syncwarp();
+        tc_fence_after_sync();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
 }
 
 // rows of at least 128 columns, whole blocks of 1024 rows
