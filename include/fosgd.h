@@ -245,7 +245,7 @@ const char* fosgd_trace_label(int k);   /* e.g. "col10:f32->ws@4", "row14:ws->pa
  *                        memory per tile and worker (tcgen05 kind::f16), and H_32, flip and the sum over
  *                        the workers in registers, instead of fp32 butterflies on the plain ALUs.
  * Either way the results are the same bit for bit (all values are integers below 2^24 in magnitude).
- * Default: FOSGD_TC_CONTIGUOUS (the choices measured faster on a B200).  Process-wide; returns the
+ * Default: both (each measured faster than its plain-ALU kernel on a B200).  Process-wide; returns the
  * previous mask. */
 enum { FOSGD_TC_STRIDED = 1, FOSGD_TC_CONTIGUOUS = 2 };
 int fosgd_set_tensor_core_pass(int mask);

@@ -179,9 +179,9 @@ Rng make_rng(uint64_t seed, uint64_t step)
     return r;
 }
 
-// which kernel runs the ten strided stages of a decoder whose source is one packed plane: 0 = packed
-// fp16 arithmetic on the plain ALUs (the faster one as measured, hence the default), 1 = tensor cores
-std::atomic<int> g_tensor_core_pass{FOSGD_TC_CONTIGUOUS};
+// which passes of a decoder whose source is one packed plane run on the tensor cores (FOSGD_TC_* bits;
+// both by default: each measured faster than its plain-ALU kernel)
+std::atomic<int> g_tensor_core_pass{FOSGD_TC_STRIDED | FOSGD_TC_CONTIGUOUS};
 bool tc_enabled() { return (g_tensor_core_pass.load(std::memory_order_relaxed) & FOSGD_TC_STRIDED) != 0; }
 bool tc_row_enabled() { return (g_tensor_core_pass.load(std::memory_order_relaxed) & FOSGD_TC_CONTIGUOUS) != 0; }
 // whether an encoder of ten strided stages + a 2^14 tile runs as the one-kernel form or as two kernels (default:

@@ -43,9 +43,10 @@ constexpr uint32_t kBOperandBytes = 8 * 2064;                 // eight column gr
 constexpr uint32_t kOffA = 0;                                 // H_128 as int8, K-major core matrices: 16 KiB
 constexpr uint32_t kOffB = 16384;                             // eight B operands
 constexpr uint32_t kOffBits = kOffB + 8 * kBOperandBytes;     // the tile's packed rows: 1024 x 16 B
-constexpr uint32_t kOffLut = kOffBits + 16384;                // byte -> eight bytes of {0, 1}: 2 KiB
-constexpr uint32_t kOffBar = kOffLut + 2048;                  // eleven mbarriers, stop word, tensor-memory base address
-constexpr uint32_t kPatchPitch = 80;                          // bytes per row of a warp's output patch: 32 fp16 + 16 (rows land on different banks)
+constexpr uint32_t kOffBar = kOffBits + 16384;                // eleven mbarriers, stop word, tensor-memory base address
+constexpr uint32_t kPatchPitch = 64;                          // bytes per row of a warp's output patch: 32 fp16; the 16-byte chunks of a row are
+                                                              // permuted by (row >> 1) & 3, which keeps both the row-wise writes and the
+                                                              // eight-rows-by-64-bytes reads off each other's banks
 constexpr uint32_t kOffPatch = kOffBar + 128;                 // one patch of 32 rows per worker warp
 constexpr uint32_t kTcSmemBytes = kOffPatch + kWorkerWarps * 32 * kPatchPitch;
 
@@ -123,18 +124,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_col_kernel(const PassParams 
     uint64_t* const bar = reinterpret_cast<uint64_t*>(smem + kOffBar);
     volatile int* const s_stop = reinterpret_cast<volatile int*>(smem + kOffBar + 96);
     uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 100);
-    const uint2* const lut = reinterpret_cast<const uint2*>(smem + kOffLut);
 
-    // ---- once per block: expansion table, the constant operand, barriers, tensor memory ----
-    if (tid < 256) {
-        uint32_t lo = 0, hi = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            lo |= (((uint32_t)tid >> j) & 1u) << (8 * j);
-            hi |= (((uint32_t)tid >> (4 + j)) & 1u) << (8 * j);
-        }
-        reinterpret_cast<uint2*>(smem + kOffLut)[tid] = make_uint2(lo, hi);
-    }
+    // ---- once per block: the constant operand, barriers, tensor memory ----
     if (tid < kWorkers) {
         // A[m][k] = (-1)^popcount(m & k): row m, 32 of its k per thread; core matrix = 8 rows x 16 bytes
         const uint32_t m = (uint32_t)tid >> 2, kc0 = ((uint32_t)tid & 3u) * 2u;
@@ -259,8 +250,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_col_kernel(const PassParams 
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     const uint32_t hw = *reinterpret_cast<const uint16_t*>(smem + kOffBits + ((uint32_t)t * 128u + kr) * 16u + cg * 2u);
-                    const uint2 a = lut[hw & 0xFFu], b = lut[hw >> 8];
-                    x[t][0] = a.x; x[t][1] = a.y; x[t][2] = b.x; x[t][3] = b.y;
+                    // four bits -> four bytes of {0, 1}: the multiplier puts bit i of the nibble at bit 8 i (its four copies of the
+                    // nibble, shifted by 0, 7, 14 and 21, do not overlap, so nothing carries); a table in shared memory cost
+                    // more than it saved (random addresses: bank conflicts on a path that is bound by shared-memory traffic)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) x[t][q] = (((hw >> (4 * q)) & 15u) * 0x00204081u) & 0x01010101u;
                 }
 #pragma unroll
                 for (int s = 0; s < 3; ++s) {
@@ -310,13 +304,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_col_kernel(const PassParams 
                         const __half2 hh = __hfma2(*reinterpret_cast<const __half2*>(&hb), two, off);
                         w[q] = *reinterpret_cast<const uint32_t*>(&hh);
                     }
-                    *reinterpret_cast<uint4*>(patch + lane * kPatchPitch + q4 * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4*>(patch + lane * kPatchPitch + (((uint32_t)q4 ^ ((lane >> 1) & 3u)) * 16u)) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
                 __syncwarp();
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const uint32_t r = 8u * i + (lane >> 2), c = lane & 3u;
-                    const uint4 q = *reinterpret_cast<const uint4*>(patch + r * kPatchPitch + c * 16u);
+                    const uint4 q = *reinterpret_cast<const uint4*>(patch + r * kPatchPitch + ((c ^ ((r >> 1) & 3u)) * 16u));
                     __stcg(reinterpret_cast<uint4*>(dst + (size_t)((uint32_t)t * 128u + lq * 32u + r) * step + c * 8u), q);   // L2 only: read next by another kernel
                 }
                 __syncwarp();
