@@ -469,6 +469,19 @@ static cudaError_t launch_col_one(const PassParams& p, cudaStream_t s)
             const cudaError_t e = launch_col4(p, s, &launched);
             if (e != cudaSuccess || launched) return e;
         }
+        if constexpr (A == 10 && (SRC == SRC_G16 || SRC == SRC_BITS)) {
+            // Rows a megabyte or more apart (the top pass of a transform longer than 2^30): 32-column tiles, so
+            // that a row visit moves 64 bytes of bf16 in and 128 bytes of fp32 out instead of half of that.
+            if (p.lo_log >= 20) {
+                auto wide = col_tile_kernel<A, SRC>;
+                constexpr size_t wsmem = (size_t)(1 << A) * 32 * 4;
+                cudaError_t e = cudaFuncSetAttribute(wide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem);
+                if (e != cudaSuccess) return e;
+                const dim3 grid((unsigned)((p.dp >> A) / 32), (unsigned)p.nworkers);
+                wide<<<grid, 1 << A, wsmem, s>>>(p);
+                return cudaGetLastError();
+            }
+        }
         auto kern = col_tile16_kernel<A, SRC>;
         constexpr size_t smem = (size_t)phys16((1 << A) * 16) * 4;
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

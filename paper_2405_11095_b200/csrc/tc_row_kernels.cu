@@ -94,14 +94,17 @@ __device__ __forceinline__ bool mbar_wait_or_stop(uint64_t* bar, uint32_t parity
     return false;
 }
 
-// 32 consecutive accumulator columns of this thread's lane: the load is asynchronous; the registers may be
-// read after tmem_load32_wait, which names them so that no use can be scheduled before it.
-__device__ __forceinline__ void tmem_load32_issue(uint32_t taddr, uint32_t (&u)[32])
+// 32 consecutive accumulator columns of this thread's lane.  The load is asynchronous: it and its wait
+// are one statement, so that the compiler never sees the destination registers as live while the load is
+// still in flight (a version that started the load earlier, underneath the staging of the next item, had
+// them spilled in between and returned stale values).
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t (&u)[32])
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
         : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
           "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
           "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
@@ -109,14 +112,10 @@ __device__ __forceinline__ void tmem_load32_issue(uint32_t taddr, uint32_t (&u)[
         : "r"(taddr) : "memory");
 }
 
-__device__ __forceinline__ void tmem_load32_wait(uint32_t (&u)[32])
+// x with its sign flipped iff the top bit of w is set
+__device__ __forceinline__ float flip_top(float x, uint32_t w)
 {
-    asm volatile("tcgen05.wait::ld.sync.aligned;"
-                 : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]),
-                   "+r"(u[8]), "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15]),
-                   "+r"(u[16]), "+r"(u[17]), "+r"(u[18]), "+r"(u[19]), "+r"(u[20]), "+r"(u[21]), "+r"(u[22]), "+r"(u[23]),
-                   "+r"(u[24]), "+r"(u[25]), "+r"(u[26]), "+r"(u[27]), "+r"(u[28]), "+r"(u[29]), "+r"(u[30]), "+r"(u[31])
-                 :: "memory");
+    return __uint_as_float(__float_as_uint(x) ^ (w & 0x80000000u));
 }
 
 __device__ __forceinline__ void hbutterfly(uint4& a, uint4& b)
@@ -320,15 +319,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
             advance(c_drain);
             if (!mbar_wait_or_stop(bar + BAR_ACC_FULL + b, u & 1u, s_stop)) return false;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            uint32_t raw[32];
-            tmem_load32_issue(tmem_base + ((lq * 32u) << 16) + b * 128u + cw * 32u, raw);
-            if (!mbar_wait_or_stop(bar + BAR_FLIPS + b, u & 1u, s_stop)) {
-                tmem_load32_wait(raw);
-                return false;
-            }
+            if (!mbar_wait_or_stop(bar + BAR_FLIPS + b, u & 1u, s_stop)) return false;
             const uint32_t fw = reinterpret_cast<const uint32_t*>(smem + kOffFlips + b * 2048u)[jrow * 4u + cw];
             const float wamp = (p.amp_mode == AMP_WEIGHT) ? amplitude_at(p, n, tile_base) : 1.f;
-            tmem_load32_wait(raw);
+            uint32_t raw[32];
+            tmem_load32(tmem_base + ((lq * 32u) << 16) + b * 128u + cw * 32u, raw);
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(bar + BAR_ACC_FREE + b);
@@ -338,10 +333,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
             butterflies32<31>(v);
             if (p.amp_mode == AMP_WEIGHT) {
 #pragma unroll
-                for (int r = 0; r < 32; ++r) accv[r] = fmaf(flip_by_bit(v[r], fw, r), wamp, accv[r]);
+                for (int r = 0; r < 32; ++r) accv[r] = fmaf(flip_top(v[r], fw << (31 - r)), wamp, accv[r]);
             } else {
 #pragma unroll
-                for (int r = 0; r < 32; ++r) accv[r] += flip_by_bit(v[r], fw, r);
+                for (int r = 0; r < 32; ++r) accv[r] += flip_top(v[r], fw << (31 - r));
             }
             if (n == W - 1) {
                 // the tile's sum is complete: scale and store 32 consecutive coordinates
