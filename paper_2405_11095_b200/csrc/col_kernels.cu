@@ -469,9 +469,10 @@ static cudaError_t launch_col_one(const PassParams& p, cudaStream_t s)
             const cudaError_t e = launch_col4(p, s, &launched);
             if (e != cudaSuccess || launched) return e;
         }
-        if constexpr (A == 10 && (SRC == SRC_G16 || SRC == SRC_BITS)) {
-            // Rows a megabyte or more apart (the top pass of a transform longer than 2^30): 32-column tiles, so
-            // that a row visit moves 64 bytes of bf16 in and 128 bytes of fp32 out instead of half of that.
+        if constexpr (A == 10 && SRC == SRC_G16) {
+            // bf16 gradients with rows megabytes apart (the top pass of a transform longer than 2^30): 32-column
+            // tiles, so that a row visit moves 64 bytes in and 128 bytes out instead of half of that (31.2 against
+            // 35.4 ms on 8 workers of 2^31; the same tiles from packed bits were slower, 30.7 against 28.0 ms)
             if (p.lo_log >= 20) {
                 auto wide = col_tile_kernel<A, SRC>;
                 constexpr size_t wsmem = (size_t)(1 << A) * 32 * 4;
