@@ -36,11 +36,11 @@
  *   - `ws` is scratch, contents undefined on entry and exit.  fosgd_workspace_bytes gives
  *     the minimum (one worker in flight); the calls that take several workers batch as many
  *     per launch as a larger `ws` allows.  Transforms that fit one thread block's tile
- *     (length <= 2^15) need none (ws may be NULL, ws_bytes 0).  The one-kernel encoder (see
- *     fosgd_set_fused_encoder) keeps 16 + 4 bytes per worker of progress words behind the
- *     intermediates: with FOSGD_FUSED_SYNC_BYTES(M) more than M times the minimum all M
- *     workers go in one launch, with exactly M times the minimum the last worker gets a
- *     launch of its own.
+ *     (length <= 2^15) need none (ws may be NULL, ws_bytes 0).  The optional one-kernel
+ *     encoder (fosgd_set_fused_encoder) keeps 16 + 4 bytes per worker of progress words
+ *     behind the intermediates: with FOSGD_FUSED_SYNC_BYTES(M) more than M times the minimum
+ *     all M workers go in one launch, with exactly M times the minimum the last worker
+ *     gets a launch of its own.
  *   - Return value: FOSGD_OK or a negative status.  On an argument, alignment, workspace,
  *     size or limit error (every status but FOSGD_ECUDA) nothing has been enqueued.
  *     FOSGD_ECUDA means a launch or a runtime call failed, possibly after earlier kernels of
@@ -239,7 +239,8 @@ const char* fosgd_trace_label(int k);   /* e.g. "col10:f32->ws@4", "row14:ws->pa
  * matrix product, and on the decode side all operands are exact small integers (Def. 3.8: q_i = +-1).
  *   FOSGD_TC_STRIDED     the ten strided stages as H_8 on packed bytes plus a 128 x 128 x 128 8-bit integer
  *                        product per block (tcgen05 kind::i8), instead of packed fp16 arithmetic on the
- *                        plain ALUs;
+ *                        plain ALUs (launches of fewer than 256 tiles of 2^17 coordinates stay on the
+ *                        plain ALUs: too few tiles to repay a block's set-up);
  *   FOSGD_TC_CONTIGUOUS  the contiguous pass on tiles of 2^14 (transform length 2^24) as H_4 in packed
  *                        fp16 while staging, a 128 x 128 x 128 fp16 product with fp32 accumulators in tensor
  *                        memory per tile and worker (tcgen05 kind::f16), and H_32, flip and the sum over
@@ -251,11 +252,12 @@ enum { FOSGD_TC_STRIDED = 1, FOSGD_TC_CONTIGUOUS = 2 };
 int fosgd_set_tensor_core_pass(int mask);
 
 /* Kernel choice for the uplink encoder of fp32 gradients when the transform length is 2^24 (ten strided
- * stages, then contiguous tiles of 2^14).  With on != 0 (the default) both passes run as one persistent
- * kernel: half of every thread block stages strided tiles through the tensor copy engine while the other
- * half transforms, dithers and packs the contiguous tiles of workers whose strided pass is complete, so
- * that the memory-bound and the issue-bound half of the encoder overlap.  With on == 0 the two passes run
- * as two kernels, one after the other.  Same bits either way.  Process-wide; returns the previous setting. */
+ * stages, then contiguous tiles of 2^14).  With on == 0 (the default) the two passes run as two kernels, one
+ * after the other.  With on != 0 both run as one persistent kernel: half of every thread block stages strided
+ * tiles through the tensor copy engine while the other half transforms, dithers and packs the contiguous
+ * tiles of workers whose strided pass is complete.  Same bits either way; measured on a B200 the two kernels
+ * are the faster form, so the one-kernel form is an option, not the default.  Process-wide; returns the
+ * previous setting. */
 int fosgd_set_fused_encoder(int on);
 #define FOSGD_FUSED_SYNC_BYTES(M) ((((size_t)(M) + 4) * 4 + 15) & ~(size_t)15)
 

@@ -278,8 +278,8 @@ def set_tensor_core_pass(mask: int) -> int:
 
 
 def set_fused_encoder(on: bool) -> bool:
-    """fosgd_set_fused_encoder: run the uplink encoder of a 2^24-long transform as one kernel (True, the
-    default) or as its two passes one after the other (False); returns the previous setting."""
+    """fosgd_set_fused_encoder: run the uplink encoder of a 2^24-long transform as one kernel (True) or as
+    its two passes one after the other (False, the default and the faster form); returns the previous setting."""
     return bool(_lib.fosgd_set_fused_encoder(int(bool(on))))
 
 

@@ -81,7 +81,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// bounded wait that also gives up when the block's stop word is raised
+// bounded wait that also gives up when the block's stop word is raised (plain polling: with a suspend-time hint
+// of 20 microseconds on the try, the contiguous pass took 0.49 instead of 0.36 ms: sleeping warps wake up late)
 __device__ __forceinline__ bool mbar_wait_or_stop(uint64_t* bar, uint32_t parity, const volatile int* stop)
 {
     for (int it = 0; it < (1 << 22); ++it) {

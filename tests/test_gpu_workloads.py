@@ -327,9 +327,16 @@ def test_tensor_core_pass_matches_plain_alu_pass(F, cfg, block_log2):
         prev = F.set_tensor_core_pass(mask)
         try:
             a = torch.empty(dp, dtype=torch.float32, device=DEV)
-            F.server_aggregate(bits, d, a, lam, seed, step, block_log2=block_log2, ws=ws)
+            with F.PassTrace() as tr:
+                F.server_aggregate(bits, d, a, lam, seed, step, block_log2=block_log2, ws=ws)
             torch.cuda.synchronize()
             acc[mask] = a
+            # the kernels asked for are the ones that ran (the strided one needs 256 tiles of 2^17 to be chosen,
+            # the contiguous one tiles of 2^14: transform length 2^24)
+            ran_strided = any(lab.startswith("tc10") for lab in tr.labels)
+            ran_contiguous = any(lab.startswith("tcrow") for lab in tr.labels)
+            assert ran_strided == (bool(mask & F.TC_STRIDED) and (dp >> 17) * M >= 256), tr.labels
+            assert ran_contiguous == (bool(mask & F.TC_CONTIGUOUS) and n_eff == 1 << 24), tr.labels
         finally:
             F.set_tensor_core_pass(prev)
     for mask in acc:
