@@ -244,11 +244,13 @@ const char* fosgd_trace_label(int k);   /* e.g. "col10:f32->ws@4", "row14:ws->pa
  *   FOSGD_TC_CONTIGUOUS  the contiguous pass on tiles of 2^14 (transform length 2^24) as H_4 in packed
  *                        fp16 while staging, a 128 x 128 x 128 fp16 product with fp32 accumulators in tensor
  *                        memory per tile and worker (tcgen05 kind::f16), and H_32, flip and the sum over
- *                        the workers in registers, instead of fp32 butterflies on the plain ALUs.
+ *                        the workers in registers, instead of fp32 butterflies on the plain ALUs (launches
+ *                        that sum fewer than three workers stay on the plain ALUs, which are faster there).
+ *   FOSGD_TC_ANY_SIZE    apply the chosen passes also to launches below the size thresholds named above.
  * Either way the results are the same bit for bit (all values are integers below 2^24 in magnitude).
- * Default: both (each measured faster than its plain-ALU kernel on a B200).  Process-wide; returns the
+ * Default: FOSGD_TC_STRIDED | FOSGD_TC_CONTIGUOUS (each measured faster than its plain-ALU kernel on a B200).  Process-wide; returns the
  * previous mask. */
-enum { FOSGD_TC_STRIDED = 1, FOSGD_TC_CONTIGUOUS = 2 };
+enum { FOSGD_TC_STRIDED = 1, FOSGD_TC_CONTIGUOUS = 2, FOSGD_TC_ANY_SIZE = 4 };
 int fosgd_set_tensor_core_pass(int mask);
 
 /* Kernel choice for the uplink encoder of fp32 gradients when the transform length is 2^24 (ten strided

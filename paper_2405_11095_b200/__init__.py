@@ -267,12 +267,12 @@ def downlink_apply(down_bits, d, x, lam_s, seed, step, step_size, K=1, block_log
     return x
 
 
-TC_STRIDED, TC_CONTIGUOUS = 1, 2
+TC_STRIDED, TC_CONTIGUOUS, TC_ANY_SIZE = 1, 2, 4
 
 
 def set_tensor_core_pass(mask: int) -> int:
     """fosgd_set_tensor_core_pass: which decoder passes from one packed plane run on the tensor cores
-    (TC_STRIDED | TC_CONTIGUOUS bits; True = the strided pass only, as in its first form); returns the
+    (TC_STRIDED | TC_CONTIGUOUS bits, TC_ANY_SIZE to skip the size thresholds); returns the
     previous mask."""
     return int(_lib.fosgd_set_tensor_core_pass(int(mask)))
 

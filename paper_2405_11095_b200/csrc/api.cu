@@ -184,6 +184,7 @@ Rng make_rng(uint64_t seed, uint64_t step)
 std::atomic<int> g_tensor_core_pass{FOSGD_TC_STRIDED | FOSGD_TC_CONTIGUOUS};
 bool tc_enabled() { return (g_tensor_core_pass.load(std::memory_order_relaxed) & FOSGD_TC_STRIDED) != 0; }
 bool tc_row_enabled() { return (g_tensor_core_pass.load(std::memory_order_relaxed) & FOSGD_TC_CONTIGUOUS) != 0; }
+bool tc_any_size() { return (g_tensor_core_pass.load(std::memory_order_relaxed) & FOSGD_TC_ANY_SIZE) != 0; }
 // whether an encoder of ten strided stages + a 2^14 tile runs as the one-kernel form or as two kernels (default:
 // measured on a B200 the two kernels are the faster form)
 std::atomic<int> g_fused_encoder{0};
@@ -255,7 +256,7 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
             pc.dst_stride = g.dp;
             pc.lo_log = pl.lo[0];
             // ten stages: H_8 on packed bytes + H_128 on the tensor cores, same fp16 intermediate
-            tensor_pass = pl.A[0] == 10 && tc_enabled() && tc_col_applicable(pc);
+            tensor_pass = pl.A[0] == 10 && tc_enabled() && tc_col_applicable(pc, tc_any_size());
             if (tensor_pass) FOSGD_CUDA_OK(traced('t', pl.A[0], SRC_BITS, 4, pc, s));
             else FOSGD_CUDA_OK(traced('h', pl.A[0], SRC_BITS, 4, pc, s));
         } else {
@@ -281,7 +282,7 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
         } else {
             pr.dst = dst0 + (size_t)n0 * (size_t)p.dst_stride * sink_elem_bytes(sink);
         }
-        if (half_path && sink == SINK_FINAL && tc_row_enabled() && tc_row_applicable(pr, pl.T))
+        if (half_path && sink == SINK_FINAL && tc_row_enabled() && tc_row_applicable(pr, pl.T, tc_any_size()))
             FOSGD_CUDA_OK(traced('u', pl.T, SRC_WS16, sink, pr, s));
         else
             FOSGD_CUDA_OK(traced('r', pl.T, half_path ? (int)SRC_WS16 : (int)SRC_WS, sink, pr, s));
@@ -700,7 +701,7 @@ const char* fosgd_trace_label(int k)
 
 int fosgd_set_tensor_core_pass(int mask)
 {
-    return g_tensor_core_pass.exchange(mask & (FOSGD_TC_STRIDED | FOSGD_TC_CONTIGUOUS), std::memory_order_relaxed);
+    return g_tensor_core_pass.exchange(mask & (FOSGD_TC_STRIDED | FOSGD_TC_CONTIGUOUS | FOSGD_TC_ANY_SIZE), std::memory_order_relaxed);
 }
 
 int fosgd_set_fused_encoder(int on)

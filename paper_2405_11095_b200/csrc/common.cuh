@@ -256,10 +256,10 @@ __attribute__((visibility("hidden"))) int check_decode_args(const void* bits, in
 cudaError_t launch_row(int T, int src, int sink, const PassParams& p, cudaStream_t s);
 cudaError_t launch_col(int A, int src, const PassParams& p, cudaStream_t s);
 cudaError_t launch_colh(int A, const PassParams& p, cudaStream_t s);   // one-plane bits -> fp16 intermediate
-bool tc_col_applicable(const PassParams& p);                            // ten strided stages from one plane on the tensor cores
+bool tc_col_applicable(const PassParams& p, bool any_size);                            // ten strided stages from one plane on the tensor cores
 cudaError_t launch_tc_col(const PassParams& p, cudaStream_t s);          // one-plane bits -> fp16 intermediate
 cudaError_t tc_timeouts(int* out);
-bool tc_row_applicable(const PassParams& p, int T);                     // contiguous 2^14 tiles of the fp16 intermediate, seven stages on the tensor cores
+bool tc_row_applicable(const PassParams& p, int T, bool any_size);                     // contiguous 2^14 tiles of the fp16 intermediate, seven stages on the tensor cores
 cudaError_t launch_tc_row(const PassParams& p, cudaStream_t s);          // fp16 intermediate -> flip + sum sink
 cudaError_t tcrow_timeouts(int* out);
 // uplink encoder of a 2^24-long transform as one kernel (strided and contiguous pass side by side)

@@ -327,15 +327,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_col_kernel(const PassParams 
 // constant operand and tensor memory before its first tile, so launches of fewer than 256 tiles (the server's
 // own vector of a 2^24 transform, everything at 2^20) are left to the packed-fp16 kernel, which is as fast or
 // faster there (0.009 against 0.017 ms on one vector of 2^20).
-bool tc_col_applicable(const PassParams& p)
+bool tc_col_applicable(const PassParams& p, bool any_size)
 {
-    return p.P == 1 && p.lo_log >= 7 && (p.dp >> (p.lo_log + 10)) >= 1 && (p.dp >> 17) * p.nworkers >= 256;
+    return p.P == 1 && p.lo_log >= 7 && (p.dp >> (p.lo_log + 10)) >= 1 && (any_size || (p.dp >> 17) * p.nworkers >= 256);
 }
 
 // Ten strided stages from one packed plane into the fp16 intermediate.
 cudaError_t launch_tc_col(const PassParams& p, cudaStream_t s)
 {
-    if (!tc_col_applicable(p)) return cudaErrorInvalidValue;
+    if (!tc_col_applicable(p, true)) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(tc_col_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 0;

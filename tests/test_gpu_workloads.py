@@ -323,7 +323,7 @@ def test_tensor_core_pass_matches_plain_alu_pass(F, cfg, block_log2):
     lam = 0.37
     ws = torch.empty(F.workspace_bytes(F.OP_AGGREGATE, d, block_log2=block_log2) * M, dtype=torch.uint8, device=DEV)
     acc = {}
-    for mask in (0, F.TC_STRIDED, F.TC_CONTIGUOUS, F.TC_STRIDED | F.TC_CONTIGUOUS):
+    for mask in (0, F.TC_STRIDED, F.TC_CONTIGUOUS, F.TC_STRIDED | F.TC_CONTIGUOUS, F.TC_STRIDED | F.TC_CONTIGUOUS | F.TC_ANY_SIZE):
         prev = F.set_tensor_core_pass(mask)
         try:
             a = torch.empty(dp, dtype=torch.float32, device=DEV)
@@ -335,8 +335,9 @@ def test_tensor_core_pass_matches_plain_alu_pass(F, cfg, block_log2):
             # the contiguous one tiles of 2^14: transform length 2^24)
             ran_strided = any(lab.startswith("tc10") for lab in tr.labels)
             ran_contiguous = any(lab.startswith("tcrow") for lab in tr.labels)
-            assert ran_strided == (bool(mask & F.TC_STRIDED) and (dp >> 17) * M >= 256), tr.labels
-            assert ran_contiguous == (bool(mask & F.TC_CONTIGUOUS) and n_eff == 1 << 24), tr.labels
+            anysz = bool(mask & F.TC_ANY_SIZE)
+            assert ran_strided == (bool(mask & F.TC_STRIDED) and (anysz or (dp >> 17) * M >= 256)), tr.labels
+            assert ran_contiguous == (bool(mask & F.TC_CONTIGUOUS) and n_eff == 1 << 24 and (anysz or M >= 3)), tr.labels
         finally:
             F.set_tensor_core_pass(prev)
     for mask in acc:
@@ -365,7 +366,8 @@ def test_tensor_core_contiguous_pass_sinks(F):
     amp_s = torch.tensor([0.75], dtype=torch.float32, device=DEV)
     x0 = torch.randn(d, generator=torch.Generator(device=DEV).manual_seed(1), device=DEV)
     res = {}
-    for mask in (0, F.TC_CONTIGUOUS):
+    TC = F.TC_CONTIGUOUS | F.TC_ANY_SIZE      # also for the one- and two-worker launches below
+    for mask in (0, TC):
         prev = F.set_tensor_core_pass(mask)
         try:
             one = torch.full((d + 64,), 7.0, dtype=torch.float32, device=DEV)
@@ -381,9 +383,9 @@ def test_tensor_core_contiguous_pass_sinks(F):
             res[mask] = (one, acc, accw, x)
         finally:
             F.set_tensor_core_pass(prev)
-    for a, b in zip(res[0], res[F.TC_CONTIGUOUS]):
+    for a, b in zip(res[0], res[TC]):
         assert torch.equal(a, b)
-    one = res[F.TC_CONTIGUOUS][0]
+    one = res[TC][0]
     assert bool((one[d:] == 7.0).all())                       # nothing written beyond the d outputs
     assert_l2_close(one[:d].cpu().numpy(), oracle.decode_full(words[1], d, seed, step, 1, lam)[:d])
     assert F.async_timeouts() == 0
