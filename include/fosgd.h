@@ -195,6 +195,20 @@ int fosgd_downlink_apply(const uint32_t* down_bits, int64_t d, uint64_t seed, ui
                          const float* lambda_s_dev, int per_block, int K, int block_log2, float step_size,
                          float* x, void* ws, size_t ws_bytes, fosgd_stream stream);
 
+/* fosgd_amplitudes (one amplitude for all workers, per_block = 0) and fosgd_encode_dev in one call, for the
+ * usual case that the gradients just encoded are the ones whose norm sets the amplitude (Theorem 5.5 with
+ * B = max_n ||g_n||_2 over the M workers of the call).  lambda_dev (and lambda_s_dev, nullable) receive the
+ * amplitudes as fosgd_amplitudes writes them; the packed signs are those of fosgd_encode_dev with that lambda.
+ * Where the first strided pass of the encoder can carry the sums (fp32 gradients, transform length 2^20 ..
+ * 2^24 in global or blocked mode, `ws` holding all M workers) the gradients are read once instead of twice;
+ * elsewhere the call runs the two calls one after the other.  The sums are added in a fixed order, so the
+ * amplitudes are reproducible, but in another order than fosgd_amplitudes uses: the two may differ in the
+ * last bit.  amp_ws: scratch of fosgd_workspace_bytes(FOSGD_OP_AMPLITUDES, ..., M, ...) bytes. */
+int fosgd_encode_measured(const void* grads, int dtype, int64_t d, int64_t worker_stride, int M, uint32_t worker_id0,
+                          uint64_t seed, uint64_t step, double alpha, double alpha_s, int block_log2, float* lambda_dev,
+                          float* lambda_s_dev, uint32_t* bits, void* ws, size_t ws_bytes, void* amp_ws,
+                          size_t amp_ws_bytes, fosgd_stream stream);
+
 /* fosgd_decode without a scratch argument (the paper has no counterpart; it computes exactly
  * what fosgd_decode computes).  For callers that must not allocate device memory where they
  * decode (no allocator reachable from their code, cudaMalloc banned because it synchronises,

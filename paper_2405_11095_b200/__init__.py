@@ -27,7 +27,7 @@ EXPORTS = ("fosgd_padded_dim", "fosgd_planes", "fosgd_lambda", "fosgd_lambda_ser
            "fosgd_trace_label", "fosgd_decode_noalloc", "fosgd_async_timeouts", "fosgd_amplitudes",
            "fosgd_encode_dev", "fosgd_server_aggregate_dev", "fosgd_downlink_decode_dev", "fosgd_downlink_apply",
            "fosgd_downlink_encode", "fosgd_probe_issue_rate", "fosgd_set_tensor_core_pass",
-           "fosgd_set_fused_encoder")
+           "fosgd_set_fused_encoder", "fosgd_encode_measured")
 
 
 class FosgdError(RuntimeError):
@@ -70,6 +70,7 @@ def _load() -> C.CDLL:
     L.fosgd_probe_issue_rate.argtypes = [cint, cint, C.POINTER(dbl), vp, vp]
     L.fosgd_set_tensor_core_pass.argtypes, L.fosgd_set_tensor_core_pass.restype = [cint], cint
     L.fosgd_set_fused_encoder.argtypes, L.fosgd_set_fused_encoder.restype = [cint], cint
+    L.fosgd_encode_measured.argtypes = [vp, cint, i64, i64, cint, u32, u64, u64, dbl, dbl, cint, vp, vp, vp, vp, sz, vp, sz, vp]
     L.fosgd_strerror.argtypes, L.fosgd_strerror.restype = [cint], C.c_char_p
     L.fosgd_last_cuda_error.restype = cint
     L.fosgd_version.restype = C.c_char_p
@@ -226,6 +227,18 @@ def encode_dev(grads, d, bits, lam, seed, step, worker_id0=0, block_log2=0, per_
     _check(_lib.fosgd_encode_dev(_ptr(grads), _dtype_code(grads), d, stride, M, worker_id0, seed, step,
                                  _ptr(lam), int(per_block), block_log2, _ptr(bits), _ptr(ws), _nbytes(ws), _stream()),
            "fosgd_encode_dev")
+    return bits
+
+
+def encode_measured(grads, d, bits, lam, lam_s, seed, step, alpha=2.0, alpha_s=2.0, worker_id0=0, block_log2=0, ws=None,
+                    amp_ws=None, worker_stride=None):
+    """fosgd_encode_measured: amplitudes(...) and encode_dev(...) in one call (one amplitude for all workers);
+    the gradients are read once where the encoder's first pass can carry the norm.  lam, lam_s: device [1]."""
+    M = grads.shape[0] if grads.dim() == 2 else 1
+    stride = worker_stride if worker_stride is not None else (grads.stride(0) if grads.dim() == 2 else d)
+    _check(_lib.fosgd_encode_measured(_ptr(grads), _dtype_code(grads), d, stride, M, worker_id0, seed, step, alpha, alpha_s,
+                                      block_log2, _ptr(lam), _ptr(lam_s), _ptr(bits), _ptr(ws), _nbytes(ws), _ptr(amp_ws),
+                                      _nbytes(amp_ws), _stream()), "fosgd_encode_measured")
     return bits
 
 

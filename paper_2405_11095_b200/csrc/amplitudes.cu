@@ -204,4 +204,12 @@ cudaError_t launch_amplitudes(const void* grads, int bf16, int64_t d, int64_t wo
     return cudaGetLastError();
 }
 
+// the second step alone: amplitudes from partial sums of squares that another kernel gathered ([M][nparts])
+cudaError_t launch_amplitudes_finalize(const double* partial, int M, int nparts, double alpha, double alpha_s, double n_eff,
+                                       float* lam, float* lam_s, cudaStream_t s)
+{
+    amplitudes_finalize_kernel<<<1, 256, 0, s>>>(partial, M, nparts, alpha, alpha_s, n_eff, lam, lam_s);
+    return cudaGetLastError();
+}
+
 }  // namespace fosgd

@@ -630,6 +630,60 @@ int fosgd_amplitudes(const void* grads, int dtype, int64_t d, int64_t worker_str
     return FOSGD_OK;
 }
 
+int fosgd_encode_measured(const void* grads, int dtype, int64_t d, int64_t worker_stride, int M, uint32_t worker_id0,
+                          uint64_t seed, uint64_t step, double alpha, double alpha_s, int block_log2, float* lambda_dev,
+                          float* lambda_s_dev, uint32_t* bits, void* ws, size_t ws_bytes, void* amp_ws,
+                          size_t amp_ws_bytes, fosgd_stream stream)
+{
+    int st = check_grad_args(grads, dtype, d, worker_stride, M, block_log2);
+    if (st != FOSGD_OK) return st;
+    if (lambda_dev == nullptr || bits == nullptr || !(alpha > 0.0) || !(alpha_s > 0.0) || !isfinite(alpha) || !isfinite(alpha_s))
+        return FOSGD_EINVAL;
+    if (!aligned16(bits) || (ws && !aligned16(ws)) || (amp_ws && !aligned16(amp_ws))) return FOSGD_EALIGN;
+    Geometry g;
+    if (!make_geometry(d, block_log2, &g)) return FOSGD_EUNSUPPORTED;
+    if (amp_ws == nullptr || amp_ws_bytes < (size_t)M * 256 * sizeof(double)) return FOSGD_EWORKSPACE;
+    if (g.plan.ncol > 0 && (ws == nullptr || ws_bytes < g.ws_per_worker)) return FOSGD_EWORKSPACE;
+    const Plan& pl = g.plan;
+    cudaStream_t s = (cudaStream_t)stream;
+    // One pass over the gradients where the strided pass can carry the sums: fp32, ten strided stages through the
+    // copy engine, and scratch for all M workers at once (the amplitude is a maximum over all of them, so every
+    // strided pass must be over before the first dither).
+    if (dtype == FOSGD_F32 && pl.ncol == 1 && pl.A[0] == 10 && ws_bytes / g.ws_per_worker >= (size_t)M) {
+        PassParams pc{};
+        pc.src = grads; pc.src_stride = worker_stride; pc.d = d; pc.dp = g.dp;
+        pc.dst = ws; pc.dst_stride = g.dp; pc.lo_log = pl.lo[0];
+        pc.P = 1; pc.K = 1; pc.nworkers = M; pc.id0 = worker_id0; pc.rng = make_rng(seed, step);
+        bool launched = false;
+        int nruns = 0;
+        bool on = trace_begin(s);
+        cudaError_t e = launch_col4_norm(pc, static_cast<double*>(amp_ws), s, &launched, &nruns);
+        if (launched) trace_end(on, s, TraceEntry{'c', pl.A[0], SRC_G32, SINK_WS, M, false});
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
+        if (launched) {
+            on = trace_begin(s);
+            e = launch_amplitudes_finalize(static_cast<const double*>(amp_ws), M, nruns, alpha, alpha_s,
+                                           (double)((int64_t)1 << g.L), lambda_dev, lambda_s_dev, s);
+            trace_end(on, s, TraceEntry{'n', g.L, 0, 5, M, false});
+            if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
+            PassParams pr = pc;
+            pr.src = ws; pr.src_stride = g.dp;
+            pr.dst = bits; pr.dst_stride = g.dp >> 5;
+            pr.dither_c = (float)(g.rootn / 16777216.0);
+            set_amp(&pr, Amp{1.f, lambda_dev, 0, 31}, AMP_DITHER);
+            e = traced('r', pl.T, SRC_WS, SINK_PACK1, pr, s);
+            if (e != cudaSuccess) { g_last_cuda_error = (int)e; return FOSGD_ECUDA; }
+            return FOSGD_OK;
+        }
+    }
+    // elsewhere: the norm pass, then the encoder
+    st = fosgd_amplitudes(grads, dtype, d, worker_stride, M, alpha, alpha_s, block_log2, 0, lambda_dev, lambda_s_dev,
+                          amp_ws, amp_ws_bytes, stream);
+    if (st != FOSGD_OK) return st;
+    return fosgd_encode_dev(grads, dtype, d, worker_stride, M, worker_id0, seed, step, lambda_dev, 0, block_log2, bits,
+                            ws, ws_bytes, stream);
+}
+
 const char* fosgd_strerror(int status)
 {
     switch (status) {

@@ -60,9 +60,12 @@ struct Col4 {
 // One run: tiles seg0 .. seg0 + 7 (16-column segments of the matrix view) of worker n, by the 512 threads
 // of a block or group (tid = 0 .. 511).  timeouts: device counter bumped when a bounded wait gave up;
 // the return value says whether the run completed (the same for all threads).
-template <typename S>
+// NORM: also add up the squares of the run's gradient entries (fp32 within a tile, fp64 across tiles and threads,
+// fixed order) and leave the sum in *run_sumsq, so that a norm needs no second pass over the gradients.
+template <typename S, bool NORM = false>
 __device__ __forceinline__ bool col4_run(const PassParams& p, const CUtensorMap* tmap, const uint32_t full_rows, const int n,
-                                         const uint32_t seg0, unsigned char* smem_raw, const int tid, int* timeouts)
+                                         const uint32_t seg0, unsigned char* smem_raw, const int tid, int* timeouts,
+                                         double* run_sumsq = nullptr)
 {
     using C = Col4;
     constexpr int A = C::A, ROWS = C::ROWS, RUN = C::RUN, NBUF = C::NBUF;
@@ -86,6 +89,7 @@ __device__ __forceinline__ bool col4_run(const PassParams& p, const CUtensorMap*
 
     int issued = 0, taken = 0;   // thread 0 only
     bool completed = true;
+    double sumsq = 0.0;
     auto issue = [&](int t) {
         uint64_t* const bar_full = full + (t % NBUF);
         const uint32_t dst0 = smem_u32(land0 + (t % NBUF) * LAND_BYTES);
@@ -145,6 +149,15 @@ __device__ __forceinline__ bool col4_run(const PassParams& p, const CUtensorMap*
                 v[4 * g + 0] = flip_at(q.x, w, sh); v[4 * g + 1] = flip_at(q.y, w, sh - 1u);
                 v[4 * g + 2] = flip_at(q.z, w, sh - 2u); v[4 * g + 3] = flip_at(q.w, w, sh - 3u);
             }
+            if (NORM) {
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    s0 = fmaf(v[4 * g + 0], v[4 * g + 0], s0); s1 = fmaf(v[4 * g + 1], v[4 * g + 1], s1);
+                    s2 = fmaf(v[4 * g + 2], v[4 * g + 2], s2); s3 = fmaf(v[4 * g + 3], v[4 * g + 3], s3);
+                }
+                sumsq += (double)((s0 + s1) + (s2 + s3));
+            }
             butterflies32<28>(v);
 #pragma unroll
             for (int g = 0; g < 8; ++g) {
@@ -198,6 +211,19 @@ __device__ __forceinline__ bool col4_run(const PassParams& p, const CUtensorMap*
         for (int k = taken; k < issued; ++k) mbar_wait(full + (k % NBUF), (uint32_t)((k / NBUF) & 1));
 #pragma unroll
         for (int b = 0; b < NBUF; ++b) mbar_inval(full + b);
+    }
+    if (NORM) {
+        // lanes, then warps, in a fixed order (the flips are no longer needed: their space holds the warps' sums)
+#pragma unroll
+        for (int s = 16; s >= 1; s >>= 1) sumsq += __shfl_xor_sync(0xFFFFFFFFu, sumsq, s);
+        double* const wsum = reinterpret_cast<double*>(flips);
+        if ((tid & 31) == 0) wsum[tid >> 5] = sumsq;
+        S::sync();
+        if (tid == 0) {
+            double total = 0.0;
+            for (int w = 0; w < C::THREADS / 32; ++w) total += wsum[w];
+            *run_sumsq = total;
+        }
     }
     return completed;
 }

@@ -246,6 +246,15 @@ __global__ void __launch_bounds__(512, 2) col4_kernel(const PassParams p, const 
                         (int)threadIdx.x, &g_col_wait_timeouts);
 }
 
+// the same, also leaving the sum of squares of every run's gradient entries in partial[worker * nruns + run]
+__global__ void __launch_bounds__(512, 2) col4_norm_kernel(const PassParams p, const __grid_constant__ CUtensorMap tmap,
+                                                           const int nruns, const uint32_t full_rows, double* const partial)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    col4_run<BlockSync, true>(p, &tmap, full_rows, (int)(blockIdx.x / (unsigned)nruns), (blockIdx.x % (unsigned)nruns) * 8u, smem_raw,
+                              (int)threadIdx.x, &g_col_wait_timeouts, partial + blockIdx.x);
+}
+
 __global__ void __launch_bounds__(1024, 1) col4_duo_kernel(const PassParams p, const __grid_constant__ CUtensorMap tmap,
                                                            const int nruns, const uint32_t full_rows)
 {
@@ -311,6 +320,28 @@ static cudaError_t launch_col4(const PassParams& p, cudaStream_t s, bool* launch
         col4_kernel<<<(unsigned)(nruns * p.nworkers), 512, Col4::SMEM_BYTES, s>>>(p, map, (int)nruns, (uint32_t)rows);
     }
     *launched = true;
+    return cudaGetLastError();
+}
+
+// Ten stages on fp32 gradients with the squared norm of every worker's gradient gathered on the way: run sums
+// in partial[worker][run] (*nruns_out of them per worker).  One-block-per-run form only; *launched stays false
+// where it does not apply (rows 128 KiB apart or more, rows shorter than a run, map refused).
+cudaError_t launch_col4_norm(const PassParams& p, double* partial, cudaStream_t s, bool* launched, int* nruns_out)
+{
+    constexpr int A = 10;
+    *launched = false;
+    const uint64_t S = (uint64_t)1 << p.lo_log;
+    const uint64_t rows = (uint64_t)(p.d >> p.lo_log);
+    const int64_t nsegs = (p.dp >> A) / 16;
+    const int64_t nruns = nsegs / 8;
+    if (p.lo_log >= 15 || S < 128 || nsegs % 8 != 0 || nruns * p.nworkers > 0x7FFFFFFF) return cudaSuccess;
+    CUtensorMap map;
+    if (!make_col_tensor_map(&map, p.src, S, rows, (uint64_t)p.nworkers, (uint64_t)p.src_stride)) return cudaSuccess;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(col4_norm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Col4::SMEM_BYTES)) != cudaSuccess) return e;
+    col4_norm_kernel<<<(unsigned)(nruns * p.nworkers), 512, Col4::SMEM_BYTES, s>>>(p, map, (int)nruns, (uint32_t)rows, partial);
+    *launched = true;
+    *nruns_out = (int)nruns;
     return cudaGetLastError();
 }
 

@@ -271,6 +271,9 @@ cudaError_t col_timeouts(int* out);                                      // sync
 cudaError_t launch_small(int L, int src, int sink, const PassParams& p, cudaStream_t s);
 cudaError_t launch_amplitudes(const void* grads, int bf16, int64_t d, int64_t worker_stride, int M, double alpha,
                               double alpha_s, double n_eff, float* lam, float* lam_s, double* partial, cudaStream_t s);
+cudaError_t launch_amplitudes_finalize(const double* partial, int M, int nparts, double alpha, double alpha_s, double n_eff,
+                                       float* lam, float* lam_s, cudaStream_t s);
+cudaError_t launch_col4_norm(const PassParams& p, double* partial, cudaStream_t s, bool* launched, int* nruns_out);
 cudaError_t launch_block_amplitudes(const void* grads, int bf16, int64_t d, int64_t dp, int64_t worker_stride, int M,
                                     int block_log2, double alpha, double alpha_s, float* lam, float* lam_s,
                                     double* seg, cudaStream_t st);

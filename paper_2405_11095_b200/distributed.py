@@ -64,9 +64,13 @@ def round_trip(codec, grads, d, buf: RoundTripBuffers, lam, lam_s, seed, step, *
     chunks = M_local // rows
     final_down = buf.down if world == 1 else None
     dev_amp = amps is not None
-    if dev_amp:
+    pb = dev_amp and amps.per_block
+    # one amplitude for all workers, one rank, all workers resident: the encoder measures the norms itself
+    # (fosgd_encode_measured reads the gradients once where its first pass can carry the sums)
+    measured_encode = (dev_amp and not amps.per_block and world == 1 and chunks == 1 and encode_streams <= 1
+                       and hasattr(codec, "encode_measured"))
+    if dev_amp and not measured_encode:
         # every distinct gradient is a row of `grads` (streamed workers cycle through the rows)
-        pb = amps.per_block
         codec.amplitudes(grads, d, amps.lam, amps.lam_s, alpha=amps.alpha, alpha_s=amps.alpha_s,
                          block_log2=block_log2, per_block=pb, ws=amps.ws, worker_stride=worker_stride)
         if world > 1:
@@ -81,6 +85,10 @@ def round_trip(codec, grads, d, buf: RoundTripBuffers, lam, lam_s, seed, step, *
         if encode_streams > 1 and rows >= encode_streams:
             _encode_on_streams(codec, grads, d, buf, lam, seed, step, first, block_log2, worker_stride,
                                amps, encode_streams)
+        elif measured_encode:
+            codec.encode_measured(grads, d, buf.bits, amps.lam, amps.lam_s, seed, step, alpha=amps.alpha,
+                                  alpha_s=amps.alpha_s, worker_id0=first, block_log2=block_log2, ws=buf.ws,
+                                  amp_ws=amps.ws, worker_stride=worker_stride)
         elif dev_amp:
             codec.encode_dev(grads, d, buf.bits, amps.lam, seed, step, worker_id0=first, block_log2=block_log2,
                              per_block=pb, ws=buf.ws, worker_stride=worker_stride)

@@ -427,3 +427,42 @@ def test_fused_encoder_matches_two_kernel_encoder(F, d, M, ws_workers, extra):
     n = M - 1
     ref, margin = oracle.encode(grads[n, :d].cpu().double().numpy(), seed, step, 2 + n, lam, want_margin=True)
     assert_bits_match(to_np_words(out[True][n])[None], ref, margin, lam)
+
+
+@pytest.mark.parametrize("d,M,b,dtype", [
+    ((1 << 24) - 70_001, 3, 0, torch.float32),     # strided pass carries the sums (one read of the gradients)
+    (1 << 20, 5, 0, torch.float32),
+    (3 * (1 << 20) + 5, 2, 20, torch.float32),     # blocked mode, one amplitude for all workers and blocks
+    ((1 << 16) + 3, 3, 0, torch.float32),          # nine strided stages: the two calls one after the other
+    (1 << 20, 2, 0, torch.bfloat16),               # bf16: likewise
+])
+def test_encode_measured_equals_amplitudes_then_encode(F, d, M, b, dtype):
+    """fosgd_encode_measured against fosgd_amplitudes + fosgd_encode_dev: the same amplitudes (to the last bits:
+    the sums are taken in another order), the same packed words for the amplitude it wrote, and those words
+    against the oracle."""
+    seed, step = 77, 5
+    dp = F.padded_dim(d, b)
+    stride = (d + 7) // 8 * 8
+    g = torch.Generator(device=DEV).manual_seed(d % 997 + M)
+    grads = (torch.randn(M, stride, generator=g, device=DEV) * (1 + torch.arange(M, device=DEV)[:, None])).to(dtype)
+    ws = torch.empty(max(16, F.workspace_bytes(F.OP_ENCODE, d, block_log2=b) * M), dtype=torch.uint8, device=DEV)
+    amp_ws = torch.empty(F.workspace_bytes(F.OP_AMPLITUDES, d, M=M, block_log2=b), dtype=torch.uint8, device=DEV)
+    lam1, lam_s1 = torch.zeros(1, device=DEV), torch.zeros(1, device=DEV)
+    lam2, lam_s2 = torch.zeros(1, device=DEV), torch.zeros(1, device=DEV)
+    bits1 = torch.zeros(M, dp // 32, dtype=torch.int32, device=DEV)
+    bits2 = torch.zeros(M, dp // 32, dtype=torch.int32, device=DEV)
+    F.encode_measured(grads, d, bits1, lam1, lam_s1, seed, step, alpha=2.0, alpha_s=3.0, worker_id0=4, block_log2=b, ws=ws,
+                      amp_ws=amp_ws, worker_stride=stride)
+    F.amplitudes(grads, d, lam2, lam_s2, alpha=2.0, alpha_s=3.0, block_log2=b, ws=amp_ws, worker_stride=stride)
+    F.encode_dev(grads, d, bits2, lam1, seed, step, worker_id0=4, block_log2=b, ws=ws, worker_stride=stride)
+    torch.cuda.synchronize()
+    assert abs(lam1.item() / lam2.item() - 1) < 1e-6 and abs(lam_s1.item() / lam_s2.item() - 1) < 1e-6
+    n_eff = F.transform_len(d, b)
+    x = grads[:, :d].double()
+    lam_ref = 2.0 * float(x.norm(dim=1).max()) * np.sqrt(np.log(n_eff) / n_eff)
+    assert abs(lam1.item() / lam_ref - 1) < 1e-6
+    assert torch.equal(bits1, bits2)
+    n = M - 1
+    ref, margin = oracle.encode(x[n].cpu().numpy(), seed, step, 4 + n, lam1.item(), block_log2=b, want_margin=True)
+    assert_bits_match(to_np_words(bits1[n])[None], ref, margin, lam1.item())
+    assert F.async_timeouts() == 0
