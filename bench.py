@@ -55,6 +55,8 @@ def parse_args():
                     help="run the uplink encoder of a 2^24-long transform as one kernel instead of two")
     ap.add_argument("--tensor-core-pass", type=int, default=None, choices=[0, 1, 2, 3],
                     help="decoder passes on the tensor cores: 1 = strided, 2 = contiguous, 3 = both (default: the library's)")
+    ap.add_argument("--ws-factor", type=float, default=1.0,
+                    help="scratch as a multiple of the minimum per worker (1.5: a decoder with two strided passes keeps its first pass in fp16)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-legs", action="store_true", help="skip the extra workloads, the K > 1 downlink table and the issue-rate probe")
@@ -311,7 +313,7 @@ def run_workload(env, args, w, steps, warmup, min_seconds, want_e2e):
     ws_per = F.workspace_bytes(F.OP_AGGREGATE, d, block_log2=b, K=w.K)
     ws_workers = args.ws_workers or R
     # (+ the progress words with which the one-kernel encoder takes all its workers in one launch)
-    ws = torch.empty(max(16, ws_per * ws_workers + F.fused_sync_bytes(ws_workers)), dtype=torch.uint8, device=dev) if ws_per else None
+    ws = torch.empty(max(16, int(ws_per * ws_workers * args.ws_factor) // 16 * 16 + F.fused_sync_bytes(ws_workers)), dtype=torch.uint8, device=dev) if ws_per else None
     buf = D.RoundTripBuffers(bits=torch.zeros(R, dp // 32, dtype=torch.int32, device=dev),
                              acc=torch.zeros(dp, dtype=torch.float32, device=dev),
                              down=torch.zeros(P, dp // 32, dtype=torch.int32, device=dev),

@@ -148,7 +148,7 @@ int planes(int K)
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool good_lambda(float l) { return isfinite(l) && l > 0.f; }
 
-size_t src_elem_bytes(int src) { return src == SRC_G16 ? 2 : 4; }
+size_t src_elem_bytes(int src) { return (src == SRC_G16 || src == SRC_WS16) ? 2 : 4; }
 size_t sink_elem_bytes(int) { return 4; }
 
 struct Geometry {
@@ -223,6 +223,16 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
     const uint32_t id0 = p.id0;
     // a packed one-plane source through a single strided pass stays exact in fp16 (|value| <= 2^A)
     const bool half_path = (src == SRC_BITS && p.P == 1 && pl.ncol == 1 && pl.A[0] >= 6);
+    // A packed one-plane source through two strided passes (transform length above 2^25): the first pass's output
+    // is still exact in fp16, so with room for it beside the fp32 intermediate (6 instead of 4 bytes per
+    // coordinate and worker) the first pass writes half the bytes in 256-byte rows and the second reads half.
+    bool half_first = (src == SRC_BITS && p.P == 1 && pl.ncol == 2 && pl.A[1] >= 6 && pl.A[1] <= 10 &&
+                       ws_bytes >= g.ws_per_worker + g.ws_per_worker / 2);
+    if (half_first) {
+        const size_t cap16 = ws_bytes / (g.ws_per_worker + g.ws_per_worker / 2);
+        chunk = (int)(cap16 < (size_t)total ? cap16 : (size_t)total);
+    }
+    char* const ws16 = static_cast<char*>(ws) + (size_t)chunk * g.ws_per_worker;   // (used by half_first only)
     for (int n0 = 0; n0 < total; n0 += chunk) {
         const int m = (total - n0 < chunk) ? total - n0 : chunk;
         PassParams q = p;
@@ -259,6 +269,21 @@ int run_transform(const Geometry& g, int src, int sink, PassParams p, void* ws, 
             tensor_pass = pl.A[0] == 10 && tc_enabled() && tc_col_applicable(pc, tc_any_size());
             if (tensor_pass) FOSGD_CUDA_OK(traced('t', pl.A[0], SRC_BITS, 4, pc, s));
             else FOSGD_CUDA_OK(traced('h', pl.A[0], SRC_BITS, 4, pc, s));
+        } else if (half_first) {
+            PassParams pc = q;
+            pc.src = srck;
+            pc.dst = ws16;
+            pc.dst_stride = g.dp;
+            pc.lo_log = pl.lo[1];
+            if (pl.A[1] == 10 && tc_enabled() && tc_col_applicable(pc, tc_any_size())) FOSGD_CUDA_OK(traced('t', pl.A[1], SRC_BITS, 4, pc, s));
+            else FOSGD_CUDA_OK(traced('h', pl.A[1], SRC_BITS, 4, pc, s));
+            PassParams pm = q;
+            pm.src = ws16;
+            pm.src_stride = g.dp;
+            pm.dst = ws;
+            pm.dst_stride = g.dp;
+            pm.lo_log = pl.lo[0];
+            FOSGD_CUDA_OK(traced('c', pl.A[0], SRC_WS16, SINK_WS, pm, s, true));
         } else {
             // strided passes, highest bits first: source -> ws, then ws -> ws in place
             for (int c = pl.ncol - 1; c >= 0; --c) {

@@ -29,6 +29,8 @@ __device__ __forceinline__ float col_load(const PassParams& p, const void* worke
         return (i < d32) ? __uint_as_float((uint32_t)__ldcs(static_cast<const uint16_t*>(worker_src) + i) << 16) : 0.f;
     } else if (SRC == SRC_WS) {
         return static_cast<const float*>(worker_src)[i];
+    } else if (SRC == SRC_WS16) {
+        return __half2float(static_cast<const __half*>(worker_src)[i]);
     } else {
         return plane_value(static_cast<const uint32_t*>(worker_src) + (i >> 5), p.dp >> 5, p.P, p.K, bit);
     }
@@ -37,7 +39,7 @@ __device__ __forceinline__ float col_load(const PassParams& p, const void* worke
 template <int SRC>
 __device__ __forceinline__ const void* worker_source(const PassParams& p, int n)
 {
-    const size_t es = (SRC == SRC_G16) ? 2 : 4;
+    const size_t es = (SRC == SRC_G16 || SRC == SRC_WS16) ? 2 : 4;
     return static_cast<const char*>(p.src) + (size_t)n * (size_t)p.src_stride * es;
 }
 
@@ -539,6 +541,9 @@ static cudaError_t launch_col_A(int src, const PassParams& p, cudaStream_t s)
         case SRC_G16: return launch_col_one<A, SRC_G16>(p, s);
         case SRC_BITS: return launch_col_one<A, SRC_BITS>(p, s);
         case SRC_WS: return launch_col_one<A, SRC_WS>(p, s);
+        case SRC_WS16:
+            if constexpr (A >= 6) return launch_col_one<A, SRC_WS16>(p, s);   // (second strided pass of a long decoder)
+            break;
     }
     return cudaErrorInvalidValue;
 }

@@ -466,3 +466,34 @@ def test_encode_measured_equals_amplitudes_then_encode(F, d, M, b, dtype):
     ref, margin = oracle.encode(x[n].cpu().numpy(), seed, step, 4 + n, lam1.item(), block_log2=b, want_margin=True)
     assert_bits_match(to_np_words(bits1[n])[None], ref, margin, lam1.item())
     assert F.async_timeouts() == 0
+
+
+def test_long_decoder_with_fp16_first_pass(F):
+    """A decoder with two strided passes (transform length 2^26): where the scratch holds 6 instead of 4 bytes per
+    coordinate for at least one worker, its first pass keeps its (exact) output in fp16.  Bit for bit against the fp32 route,
+    and against the oracle."""
+    d, seed, step, M = (1 << 26) - 12_345, 3, 8, 3
+    dp = F.padded_dim(d)
+    rng = np.random.default_rng(26)
+    words = rng.integers(0, 2 ** 32, (M, dp // 32), dtype=np.uint64).astype(np.uint32)
+    words[0, : dp // 64] = 0xFFFFFFFF
+    bits = torch.from_numpy(words.view(np.int32)).to(DEV)
+    lam = 0.83
+    per = F.workspace_bytes(F.OP_AGGREGATE, d)
+    acc = {}
+    # scratch for one worker in fp32 only: worker by worker on the fp32 route; 1.5 x M workers: all three at once
+    for name, nbytes in (("fp32", per), ("fp16 first", per * M * 3 // 2)):
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=DEV)
+        a = torch.empty(dp, dtype=torch.float32, device=DEV)
+        with F.PassTrace() as tr:
+            F.server_aggregate(bits, d, a, lam, seed, step, ws=ws)
+        torch.cuda.synchronize()
+        assert any("ws16->ws" in lab for lab in tr.labels) == (name == "fp16 first"), tr.labels
+        acc[name] = a
+        del ws
+    assert torch.equal(acc["fp32"], acc["fp16 first"])
+    gbar = np.zeros(dp)
+    for part in pmap(lambda n: oracle.decode_full(words[n], d, seed, step, n, lam), range(M)):
+        gbar += part
+    assert_l2_close(acc["fp16 first"].cpu().numpy(), gbar / M)
+    assert F.async_timeouts() == 0
