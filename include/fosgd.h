@@ -36,7 +36,11 @@
  *   - `ws` is scratch, contents undefined on entry and exit.  fosgd_workspace_bytes gives
  *     the minimum (one worker in flight); the calls that take several workers batch as many
  *     per launch as a larger `ws` allows.  Transforms that fit one thread block's tile
- *     (length <= 2^15) need none (ws may be NULL, ws_bytes 0).  The optional one-kernel
+ *     (length <= 2^15) need none (ws may be NULL, ws_bytes 0).  A decoder from one packed
+ *     plane whose transform is longer than 2^25 keeps the output of its first pass in fp16
+ *     beside the fp32 intermediate where `ws` has 1.5 times the minimum for at least one
+ *     worker (it then batches ws_bytes / (1.5 * minimum) workers per launch): less traffic,
+ *     same result bit for bit.  The optional one-kernel
  *     encoder (fosgd_set_fused_encoder) keeps 16 + 4 bytes per worker of progress words
  *     behind the intermediates: with FOSGD_FUSED_SYNC_BYTES(M) more than M times the minimum
  *     all M workers go in one launch, with exactly M times the minimum the last worker
