@@ -353,7 +353,7 @@ def run_workload(env, args, w, steps, warmup, min_seconds, want_e2e):
     # CUDA events around every step, per-kernel events through the library's trace hook.  Blocks
     # repeat until min_seconds of device time have been timed; the median block is reported. ----
     K = steps
-    traces = [F.PassTrace(64) for _ in range(K)]
+    traces = [F.PassTrace(256) for _ in range(K)]
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
     sampler = ClockSampler(local_rank) if rank == 0 else None
     block_ms, per, order, nblocks, timed_ms = [], {}, [], 0, 0.0

@@ -244,7 +244,7 @@ int fosgd_async_timeouts(int* count);
 /* Profiling aid (no counterpart in the paper).  events: HOST array of 2*capacity cudaEvent_t
  * handles created by the caller with timing enabled, or NULL to switch tracing off.  While set,
  * every kernel launch issued by the calling thread records events[2k] before and events[2k+1]
- * after launch number k (k < capacity, at most 64), so that cudaEventElapsedTime gives each
+ * after launch number k (k < capacity, at most 256), so that cudaEventElapsedTime gives each
  * kernel's duration.  Setting the array resets the launch counter.  Thread local. */
 int fosgd_trace_passes(void** events, int capacity);
 int fosgd_trace_count(void);            /* launches recorded since the array was set */

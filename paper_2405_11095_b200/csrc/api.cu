@@ -47,12 +47,13 @@ struct TraceEntry { char kind; int size, src, sink, workers; bool decoder; };   
 thread_local cudaEvent_t* g_trace_events = nullptr;
 thread_local int g_trace_capacity = 0;
 thread_local int g_trace_count = 0;
-thread_local TraceEntry g_trace_log[64];
+constexpr int kTraceMax = 256;
+thread_local TraceEntry g_trace_log[kTraceMax];
 thread_local char g_trace_label[48];
 
 bool trace_begin(cudaStream_t s)
 {
-    const bool on = g_trace_events != nullptr && g_trace_count < g_trace_capacity && g_trace_count < 64;
+    const bool on = g_trace_events != nullptr && g_trace_count < g_trace_capacity && g_trace_count < kTraceMax;
     if (on) cudaEventRecord(g_trace_events[2 * g_trace_count], s);
     return on;
 }
@@ -637,7 +638,7 @@ int fosgd_amplitudes(const void* grads, int dtype, int64_t d, int64_t worker_str
                                   : (size_t)M * 256 * sizeof(double);
     if (ws == nullptr || ws_bytes < need) return FOSGD_EWORKSPACE;
     if (!aligned16(ws)) return FOSGD_EALIGN;
-    const bool on = g_trace_events != nullptr && g_trace_count < g_trace_capacity && g_trace_count < 64;
+    const bool on = g_trace_events != nullptr && g_trace_count < g_trace_capacity && g_trace_count < kTraceMax;
     if (on) cudaEventRecord(g_trace_events[2 * g_trace_count], (cudaStream_t)stream);
     const cudaError_t e =
         per_block ? launch_block_amplitudes(grads, dtype == FOSGD_BF16, d, g.dp, worker_stride, M, block_log2, alpha,
