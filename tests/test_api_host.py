@@ -127,6 +127,16 @@ def test_argument_checks_return_before_any_launch(F):
     assert F.workspace_bytes(F.OP_BLOCK_AMPLITUDES, 1 << 16, M=3, block_log2=7) == 3 * 512 * 8
     assert F.workspace_bytes(F.OP_BLOCK_AMPLITUDES, 1 << 16, M=3, block_log2=12) == 3 * 64 * 8
 
+    em = lambda **k: L.fosgd_encode_measured(k.get("g", a), k.get("dt", 0), 1 << 16, 1 << 16, k.get("M", 2), 0, 1, 2,
+                                             k.get("alpha", 2.0), 2.0, 0, k.get("lam", a), a, k.get("bits", a),
+                                             k.get("ws", a), k.get("wsb", 1 << 30), k.get("aws", a), k.get("awsb", 1 << 20), None)
+    assert em(g=None) == F.EINVAL and em(lam=None) == F.EINVAL and em(bits=None) == F.EINVAL and em(alpha=-1.0) == F.EINVAL
+    assert em(dt=5) == F.EUNSUPPORTED and em(bits=a + 4) == F.EALIGN and em(aws=a + 8) == F.EALIGN
+    assert em(aws=None) == F.EWORKSPACE and em(awsb=2 * 2048 - 1) == F.EWORKSPACE
+    assert em(ws=None, wsb=0) == F.EWORKSPACE and em(wsb=100) == F.EWORKSPACE
+    assert L.fosgd_set_tensor_core_pass(L.fosgd_set_tensor_core_pass(0)) == 0        # (returns the previous mask; restored)
+    assert L.fosgd_set_fused_encoder(L.fosgd_set_fused_encoder(1)) == 1
+
     assert L.fosgd_decode_noalloc(a, (1 << 20) + 1, 0, 1, 2, 0.1, 0, a, None) == F.ELIMIT
     assert L.fosgd_decode_noalloc(a, 0, 0, 1, 2, 0.1, 0, a, None) == F.EINVAL
 
