@@ -297,6 +297,17 @@ def test_config4_bf16_1p3B_sampled(F, block_log2):
     assert abs(float(one.double().norm()) / (lam * np.sqrt(dp)) - 1) < 1e-5      # Remark 5.2: ||D(q)|| = lambda sqrt(d')
     ratio = float((one[:d].double() * x).sum() / (x * x).sum())
     assert abs(ratio - 1) < 0.05
+    if b == 0:
+        # the same decoder with 6 bytes of scratch per coordinate: first strided pass in fp16 (on the tensor cores),
+        # second one fp16 -> fp32; all values are exact integers up to the final scale, so nothing may differ
+        del x, g
+        ws6 = torch.empty(ws.numel() * 3 // 2, dtype=torch.uint8, device=DEV)
+        two = torch.empty(dp, dtype=torch.float32, device=DEV)
+        with F.PassTrace() as tr:
+            F.server_aggregate(bits[3:4], d, two, lam, seed, step, N_total=1, worker_id0=63, block_log2=b, ws=ws6)
+        torch.cuda.synchronize()
+        assert any("ws16->ws" in lab for lab in tr.labels), tr.labels
+        assert torch.equal(one, two)
 
 
 def test_no_bounded_wait_gave_up(F):
