@@ -28,7 +28,7 @@
 // next ones run.  The packed rows of the next tile are fetched into registers under the current one.
 // Synchronisation is by mbarriers (operands staged / all products of the tile done, accumulator full /
 // drained); every wait is bounded.
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace fosgd {
 
@@ -52,20 +52,9 @@ constexpr uint32_t kTcSmemBytes = kOffPatch + kWorkerWarps * 32 * kPatchPitch;
 
 enum { BAR_B_FULL = 0, BAR_B_DONE = 1, BAR_ACC_FULL = 2, BAR_ACC_FREE = 6, BAR_BITS = 10 };
 
-// shared-memory matrix descriptor, no swizzle: start address, leading and stride byte offsets in
-// units of 16 bytes, descriptor version 1
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
-           ((uint64_t)(sbo_bytes >> 4) << 32) | ((uint64_t)1 << 46);
-}
-
 // instruction descriptor: D = s32 (2 << 4), A = B = signed 8-bit (1 << 7, 1 << 10), A K-major, B MN-major
 // (1 << 16), N = 128 (N / 8 << 17), M = 128 (M / 16 << 24)
 constexpr uint32_t kIdescI8 = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (16u << 17) | (8u << 24);
-
-__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate)
 {
@@ -73,40 +62,6 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescI8), "r"(accumulate) : "memory");
-}
-
-// 32 consecutive accumulator columns of this thread's lane (load and wait in one statement: the destination
-// registers are never live while the load is in flight)
-__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t (&u)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
-          "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
-          "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
-          "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
-        : "r"(taddr) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-// bounded wait that also gives up when the block's stop word is raised
-__device__ __forceinline__ bool mbar_wait_or_stop(uint64_t* bar, uint32_t parity, const volatile int* stop)
-{
-    for (int it = 0; it < (1 << 22); ++it) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-        if (done) return true;
-        if ((it & 255) == 255 && *stop) return false;
-    }
-    return false;
 }
 
 }  // namespace
@@ -182,10 +137,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_col_kernel(const PassParams 
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)   // K = 32 per instruction: two core matrices of A, four k-groups of B
                         umma_i8(tmem_base + a * 128u, adesc + (uint64_t)(ks * (256 >> 4)), bdesc + (uint64_t)(ks * (512 >> 4)), ks > 0 ? 1u : 0u);
-                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar + BAR_ACC_FULL + a)) : "memory");
+                    umma_commit(bar + BAR_ACC_FULL + a);
                     ++issued;
                 }
-                if (ok) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar + BAR_B_DONE)) : "memory");
+                if (ok) umma_commit(bar + BAR_B_DONE);
             }
             if (!ok) {
                 if (atomicExch((int*)s_stop, 1) == 0) atomicAdd(&g_tc_wait_timeouts, 1);

@@ -24,7 +24,7 @@
 // accumulator of the previous item while the product of this one runs.  Synchronisation is by
 // mbarriers only (slot landed / read, operand full / free, accumulator full / free, flips ready);
 // every wait is bounded.
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace fosgd {
 
@@ -55,62 +55,12 @@ enum { BAR_B_FULL = 0, BAR_B_FREE = 2, BAR_ACC_FULL = 4, BAR_ACC_FREE = 6, BAR_F
 // instruction descriptor: D = f32 (1 << 4), A = B = fp16 (0), A K-major, B MN-major (1 << 16), N = 128, M = 128
 constexpr uint32_t kIdescF16 = (1u << 4) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
-// shared-memory matrix descriptor, no swizzle: start address, leading and stride byte offsets in
-// units of 16 bytes, descriptor version 1
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
-           ((uint64_t)(sbo_bytes >> 4) << 32) | ((uint64_t)1 << 46);
-}
-
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescF16), "r"(accumulate) : "memory");
-}
-
-__device__ __forceinline__ void umma_commit(uint64_t* bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-// bounded wait that also gives up when the block's stop word is raised (plain polling: with a suspend-time hint
-// of 20 microseconds on the try, the contiguous pass took 0.49 instead of 0.36 ms: sleeping warps wake up late)
-__device__ __forceinline__ bool mbar_wait_or_stop(uint64_t* bar, uint32_t parity, const volatile int* stop)
-{
-    for (int it = 0; it < (1 << 22); ++it) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-        if (done) return true;
-        if ((it & 255) == 255 && *stop) return false;
-    }
-    return false;
-}
-
-// 32 consecutive accumulator columns of this thread's lane.  The load is asynchronous: it and its wait
-// are one statement, so that the compiler never sees the destination registers as live while the load is
-// still in flight (a version that started the load earlier, underneath the staging of the next item, had
-// them spilled in between and returned stale values).
-__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t (&u)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
-          "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
-          "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
-          "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
-        : "r"(taddr) : "memory");
 }
 
 // x with its sign flipped iff the top bit of w is set
@@ -182,9 +132,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
         *s_stop = 0;
     }
     fence_generic_before_async();   // the constant operand, for the tensor core's reads
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    tc_fence_before_sync();
     __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
     const int W = p.nworkers;
@@ -216,7 +166,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
                 ok = mbar_wait_or_stop(bar + BAR_B_FULL + b, u & 1u, s_stop);                        // operand staged
                 if (ok && u > 0) ok = mbar_wait_or_stop(bar + BAR_ACC_FREE + b, (u - 1u) & 1u, s_stop);   // accumulator drained
                 if (!ok) break;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                tc_fence_after_sync();
                 const uint64_t bdesc = umma_desc(smem_u32(smem + kOffB + b * kBBytes), 128u, kBGroupStride);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)   // K = 16 per instruction: two 16-byte chunks of A, two groups of eight rows of B
@@ -319,13 +269,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
             const int64_t tile_base = c_drain.tile_base;
             advance(c_drain);
             if (!mbar_wait_or_stop(bar + BAR_ACC_FULL + b, u & 1u, s_stop)) return false;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            tc_fence_after_sync();
             if (!mbar_wait_or_stop(bar + BAR_FLIPS + b, u & 1u, s_stop)) return false;
             const uint32_t fw = reinterpret_cast<const uint32_t*>(smem + kOffFlips + b * 2048u)[jrow * 4u + cw];
             const float wamp = (p.amp_mode == AMP_WEIGHT) ? amplitude_at(p, n, tile_base) : 1.f;
             uint32_t raw[32];
             tmem_load32(tmem_base + ((lq * 32u) << 16) + b * 128u + cw * 32u, raw);
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar + BAR_ACC_FREE + b);
             float v[32];
@@ -391,11 +341,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_row_final_kernel(const PassPar
         if (ok && nitems > 0) ok = drain_item(nitems - 1);
         if (!ok && lane == 0 && atomicExch((int*)s_stop, 1) == 0) atomicAdd(&g_tcrow_wait_timeouts, 1);
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    tc_fence_before_sync();
     __syncthreads();
     if (warp == kIssueWarp) {
         __syncwarp();
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        tc_fence_after_sync();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
     }
 }
