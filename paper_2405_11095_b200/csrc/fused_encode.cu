@@ -21,10 +21,6 @@
 #include <cuda.h>
 
 #include "col4.cuh"
-
-namespace fosgd {
-static __device__ int g_async_wait_timeouts;   // named by row_kernels.cuh's streaming kernel (not used in this unit)
-}
 #include "row_kernels.cuh"
 
 namespace fosgd {

@@ -8,10 +8,6 @@
 #define FOSGD_CAT2(a, b) a##b
 #define FOSGD_CAT(a, b) FOSGD_CAT2(a, b)
 
-namespace fosgd {
-static __device__ int g_async_wait_timeouts;   // blocks of this unit that abandoned a bounded wait
-}
-
 #include "row_kernels.cuh"
 
 namespace fosgd {

@@ -357,7 +357,8 @@ __global__ void __launch_bounds__(1 << (T - 5), min_blocks<T, SINK>()) row_kerne
 // =============================================================================================
 // row_stream_kernel: tiles of an intermediate (fp32 or fp16) fetched by bulk async copies
 // =============================================================================================
-// g_async_wait_timeouts (defined by the including unit): bumped when a bounded wait on a bulk copy gave up
+// bumped when a bounded wait on a bulk copy gave up (one counter per translation unit that includes this file)
+static __device__ int g_async_wait_timeouts;
 
 // one elected thread: announce `bytes` on the barrier and start the copy global -> shared
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar)

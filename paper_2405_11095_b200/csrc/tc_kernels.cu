@@ -13,8 +13,9 @@
 //      instructions of K = 32 per product, issued by one thread, completion through an mbarrier.
 //   3. The accumulators come back with tcgen05.ld (a thread = one output row j of a lane quarter,
 //      32 columns per load), become fp16 (all values are even integers of magnitude <= 1024) and
-//      go to global memory through a padded staging tile, so that every store instruction of a
-//      warp writes two whole 256-byte rows.
+//      go to global memory through a small patch of shared memory per warp, so that a store
+//      instruction writes 64 contiguous bytes of eight rows (16 bytes per lane straight from the
+//      registers would be 32 separate requests per instruction: measured a third slower).
 // Constants: the +-1 entries are q = 2 b - 1 and the H_8 stages add byte biases 1, 2, 4, after which
 // every t' != 0 carries bias 4 and t' = 0 carries 0 but owes -8 from the "- 1".  Through the product
 // both become the same offset on output row j = 0 alone (the all-ones row of H_128): D = v / 2 + 512
@@ -24,8 +25,7 @@
 //
 // A block is 16 worker warps and one warp that issues the products, persistent over tiles.  Tensor
 // memory holds four 128-column accumulators used in turn, so that while the worker warps drain one
-// (tcgen05.ld, convert, 64 contiguous bytes per thread straight to global memory) the products of the
-// next ones run.  The packed rows of the next tile are fetched into registers under the current one.
+// (tcgen05.ld, convert, store through the warp's patch) the products of the next ones run.  The packed rows of the next tile are fetched into registers under the current one.
 // Synchronisation is by mbarriers (operands staged / all products of the tile done, accumulator full /
 // drained); every wait is bounded.
 #include "tc_common.cuh"
